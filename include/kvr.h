@@ -1,0 +1,252 @@
+/*
+ * kvr.h -- C ABI of the tiered KV-retention data mover for one GPU.
+ *
+ * The paper prices three places a suspended request's KV cache can be
+ * (Section 3.1, Eq. 1: state 1 = GPU HBM, 2 = host DRAM, 3 = discarded) and a
+ * two-stage policy that moves it between them (Section 3.4; exact semantics in
+ * Appendix D).  This library is the mechanism under that policy: a paged HBM
+ * block pool, a pinned host arena, and the moves between the two.
+ *
+ *   suspend : gather a request's scattered K/V blocks, by its block table,
+ *             into one contiguous image in pinned host memory; free the blocks
+ *   resume  : scatter the image into freshly allocated, non-contiguous blocks
+ *   retain  : leave the blocks where they are, count them as pinned
+ *   expire  : drop the host image (or the blocks); resume then answers
+ *             "recompute"
+ *
+ * Layouts (the paper leaves them open; they are fixed here):
+ *   pool  : bytes [layers][2][num_blocks][block_size][kv_heads][head_dim][dtype_bytes]
+ *           plane 0 = K, plane 1 = V; one (layer, plane, block) tile is contiguous
+ *   image : bytes [layers][2][n_tokens][kv_heads][head_dim][dtype_bytes]
+ *           exactly n_tokens * kvr_bytes_per_token() bytes, valid tokens only
+ * Bookkeeping rules (also fixed here): the free queue is FIFO (allocate from
+ * the head, release to the tail in logical block order); host ranges are
+ * placed first-fit at the lowest offset in 4096-byte granules.
+ *
+ * Conventions
+ *   - every pointer argument is a HOST pointer unless its comment says device;
+ *   - the pool handle and all metadata belong to the library; buffers passed in
+ *     kvr_config belong to the caller and must outlive the pool;
+ *   - no exceptions cross this boundary; every call returns a kvr_status:
+ *     0 = done, > 0 = a normal outcome the policy must handle, < 0 = error.
+ *     Batch calls handle the requests in the order given, each one atomically
+ *     (moved or unchanged), write each outcome to per_req (may be NULL) and
+ *     return the most negative status if any is an error, else the largest;
+ *   - moves are asynchronous: a call enqueues GPU work and returns, unless
+ *     KVR_SYNC is given.  Bookkeeping (states, block tables, arena offsets) is
+ *     final when the call returns; the bytes are final once kvr_wait() on the
+ *     request (or KVR_ALL) returns KVR_OK.  Until then kvr_request_info()
+ *     reports KVR_SUSPENDING / KVR_RESUMING.  Later calls that touch the same
+ *     blocks or host bytes are ordered after the move on the device, so the
+ *     caller never has to wait for correctness of the library's own moves;
+ *   - one caller thread per pool.
+ */
+#ifndef KVR_H
+#define KVR_H
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kvr_pool kvr_pool;
+typedef int32_t kvr_status;
+
+enum {
+  KVR_OK = 0,
+  KVR_RESIDENT = 1,      /* resume of a retained request: nothing moved (beta_1 = 0) */
+  KVR_RECOMPUTE = 2,     /* resume of an expired request: caller must re-prefill */
+  KVR_HOST_FULL = 3,     /* suspend not admitted to the host tier; request unchanged */
+  KVR_HBM_FULL = 4,      /* not enough free blocks; request unchanged */
+  KVR_ERR_INVALID_ARG = -1,
+  KVR_ERR_UNKNOWN_REQUEST = -2,
+  KVR_ERR_BAD_STATE = -3,
+  KVR_ERR_GEOMETRY = -4,
+  KVR_ERR_CUDA = -5,
+  KVR_ERR_TIMEOUT = -6,
+  KVR_ERR_NOMEM = -7
+};
+
+/* request states as reported by kvr_request_info() */
+enum {
+  KVR_ACTIVE = 0, KVR_RETAINED = 1, KVR_SUSPENDING = 2, KVR_HOST = 3, KVR_RESUMING = 4, KVR_EXPIRED = 5
+};
+
+/* call flags */
+#define KVR_SYNC 1u                  /* wait for the enqueued moves before returning */
+/* pool flags (kvr_config.flags) */
+#define KVR_METADATA_ONLY 1u         /* bookkeeping only: no buffers, no CUDA calls, nothing moves */
+#define KVR_PROFILE 2u               /* bracket every mover launch with timing events (kvr_stats.kernel_ms_*) */
+
+#define KVR_ROUTE_STAGED 1           /* kernel <-> HBM staging ring <-> chunked cudaMemcpyAsync */
+#define KVR_ROUTE_MAPPED 2           /* kernel reads / writes the pinned arena directly over the host link */
+#define KVR_KERNEL_WARP 1            /* one warp per tile, 16-byte loads and stores */
+#define KVR_KERNEL_BULK 2            /* bulk async copies through a shared-memory ring */
+
+#define KVR_ALL UINT64_MAX
+
+typedef struct {
+  int32_t layers, kv_heads, head_dim, dtype_bytes, block_size;
+} kvr_geometry;
+
+typedef struct {
+  kvr_geometry g;
+  int32_t num_blocks;
+  int32_t device;                    /* CUDA device ordinal */
+  uint64_t host_capacity_bytes;      /* host tier budget */
+  uint64_t chunk_bytes;              /* staging slot size, multiple of 4096; 0 = 64 MiB */
+  int32_t staging_slots;             /* slots per direction; 0 = 3 */
+  int32_t route;                     /* KVR_ROUTE_*; 0 = KVR_ROUTE_STAGED */
+  int32_t kernel;                    /* KVR_KERNEL_*; 0 = KVR_KERNEL_WARP */
+  int32_t max_ctas;                  /* cap on the movers' grid (0 = fill the GPU) */
+  uint32_t flags;                    /* KVR_METADATA_ONLY | KVR_PROFILE */
+  uint32_t reserved;
+  void *device_pool;                 /* DEVICE pointer to num_blocks*block_size*bytes_per_token bytes,
+                                        256-byte aligned, or NULL: the library allocates and frees it */
+  void *host_arena;                  /* page-locked HOST pointer to host_capacity_bytes bytes, 4096-byte
+                                        aligned, or NULL: the library allocates and frees it */
+  const int32_t *initial_free_order; /* permutation of [0, num_blocks) or NULL = 0, 1, 2, ... */
+} kvr_config;
+
+typedef struct {
+  int64_t blocks_total, blocks_free, blocks_active, blocks_pinned;
+  uint64_t host_capacity, host_used, host_largest_hole;
+  int64_t n_active, n_retained, n_host, n_expired;
+  int64_t suspends, resumes, resident_resumes, expires, recompute_marked;
+  int64_t host_full_rejects, hbm_full_rejects;
+  uint64_t bytes_suspended, bytes_resumed, bytes_expired_from_host;
+  /* engine counters (zero for a metadata-only pool) */
+  int64_t ops_in_flight;
+  int64_t gather_launches, scatter_launches;     /* kernel launches so far */
+  int64_t d2h_copies, h2d_copies;                /* cudaMemcpyAsync calls so far */
+  uint64_t gather_bytes, scatter_bytes;          /* payload bytes moved by the kernels */
+  uint64_t d2h_bytes, h2d_bytes;                 /* bytes moved by copies (descriptors excluded) */
+  uint64_t desc_bytes;                           /* descriptor and block-table bytes uploaded */
+  double gather_ms, scatter_ms;                  /* summed kernel durations, KVR_PROFILE only */
+} kvr_stats;
+
+/*
+ * Per-token KV bytes = 2 (K and V) x layers x kv_heads x head_dim x dtype_bytes
+ * (Appendix B, price-vector calibration: 80 x 8 x 128 x 2 x 2 = 327,680).
+ * Returns 0 for a NULL or invalid geometry (any field < 1, dtype_bytes not in
+ * {1,2,4}, or kv_heads*head_dim*dtype_bytes not a multiple of 16).
+ */
+uint64_t kvr_bytes_per_token(const kvr_geometry *g);
+
+/*
+ * Create the HBM block pool and the host tier (Appendix A: paged block pool with
+ * a free queue; Appendix D: host tier with a capacity enforced at admission).
+ * Allocates the staging rings, streams and events on cfg->device, and whichever
+ * of device_pool / host_arena is NULL.  *out is set only on KVR_OK.
+ * Errors: KVR_ERR_INVALID_ARG (NULL, bad sizes, free order not a permutation),
+ * KVR_ERR_GEOMETRY, KVR_ERR_NOMEM, KVR_ERR_CUDA.
+ */
+kvr_status kvr_pool_create(const kvr_config *cfg, kvr_pool **out);
+/* Waits for all moves in flight, then frees everything the library allocated. */
+kvr_status kvr_pool_destroy(kvr_pool *pool);
+
+/*
+ * Bring a request into the pool as ACTIVE with ceil(n_tokens/block_size) blocks
+ * from the head of the free queue (in a server the engine's own allocator does
+ * this; here it is what tests and benchmarks use).  out_blocks (cap entries,
+ * may be NULL) receives the block table.  The blocks are safe to write when the
+ * call returns: it waits for any gather still reading them.  Re-admitting an
+ * EXPIRED id is allowed (the recompute happened).  n_tokens = 0 is legal.
+ * KVR_HBM_FULL, KVR_ERR_BAD_STATE (id exists), KVR_ERR_INVALID_ARG.
+ */
+kvr_status kvr_request_admit(kvr_pool *pool, uint64_t req_id, int64_t n_tokens, int32_t *out_blocks, int32_t cap);
+/* Forget a request in any state; its blocks go to the free tail, its host range is freed. */
+kvr_status kvr_request_release(kvr_pool *pool, uint64_t req_id);
+
+/*
+ * State 1 of Eq. 1 (Section 3.1): keep the KV in HBM.  ACTIVE -> RETAINED; the
+ * blocks stay allocated and are counted in blocks_pinned (Appendix A, victim
+ * exclusion).  No data moves.  Other states: KVR_ERR_BAD_STATE.
+ */
+kvr_status kvr_retain_in_hbm(kvr_pool *pool, const uint64_t *req, int32_t n, kvr_status *per_req);
+
+/*
+ * State 1 -> 2 (Section 3.4 stage one; Appendix D: "on suspension, a context
+ * moves to host DRAM").  For each ACTIVE or RETAINED request, in order: reserve
+ * an image range in the host arena (no room: KVR_HOST_FULL, request unchanged,
+ * nobody displaced -- the replay admission rule of Appendix D), gather
+ *   image[l][kv][t][..] = pool[l][kv][table[t / block_size]][t % block_size][..]
+ * into it, and append the blocks to the free-queue tail.  Pool bytes are not
+ * scrubbed.  flags: KVR_SYNC.
+ */
+kvr_status kvr_suspend_to_host(kvr_pool *pool, const uint64_t *req, int32_t n, uint32_t flags, kvr_status *per_req);
+
+/*
+ * State 2 or 1 -> 3 (Appendix D: when the one-shot timer fires the host copy is
+ * discarded, which frees host capacity).  HOST: the image range is freed.
+ * ACTIVE / RETAINED: the blocks go to the free tail.  The request becomes
+ * EXPIRED and is counted in recompute_marked.  An EXPIRED request cannot be
+ * expired again (KVR_ERR_BAD_STATE).  No data moves.
+ */
+kvr_status kvr_expire(kvr_pool *pool, const uint64_t *req, int32_t n, kvr_status *per_req);
+
+/*
+ * Resume (Section 3.1: pays beta_2 from host, nothing from HBM, beta_3 after a
+ * discard).  HOST: take ceil(n_tokens/block_size) blocks from the free-queue
+ * head (too few: KVR_HBM_FULL, unchanged), scatter the image into them (bytes
+ * of a partial last block beyond n_tokens are not written), free the host
+ * range, -> ACTIVE.  RETAINED: -> ACTIVE, same blocks, KVR_RESIDENT.  EXPIRED:
+ * KVR_RECOMPUTE, unchanged.  ACTIVE: KVR_ERR_BAD_STATE.  flags: KVR_SYNC.
+ */
+kvr_status kvr_resume_from_host(kvr_pool *pool, const uint64_t *req, int32_t n, uint32_t flags, kvr_status *per_req);
+/*
+ * Same move for one HOST request into blocks the caller names (each currently
+ * free, no repeats, nb = its block count); the other free ids keep their
+ * order.  This is how "any block relabelling" is exercised.
+ */
+kvr_status kvr_resume_from_host_into(kvr_pool *pool, uint64_t req, const int32_t *blocks, int32_t nb, uint32_t flags);
+
+/*
+ * The two kernels on their own, HBM to HBM, no state change: write the images
+ * of n ACTIVE/RETAINED requests one after another (each start rounded up to 256
+ * bytes) into the DEVICE buffer dst, or read them back from src into the
+ * requests' current blocks.  offsets (n entries, may be NULL) receives each
+ * image's byte offset.  KVR_ERR_INVALID_ARG if capacity is too small.
+ * Used to measure and to check the gather / scatter kernels in isolation.
+ */
+kvr_status kvr_export_to_device(kvr_pool *pool, const uint64_t *req, int32_t n, void *dst_device,
+                                uint64_t capacity, uint64_t *offsets, uint32_t flags);
+kvr_status kvr_import_from_device(kvr_pool *pool, const uint64_t *req, int32_t n, const void *src_device,
+                                  uint64_t capacity, uint64_t *offsets, uint32_t flags);
+
+/*
+ * Observe one request.  Any out pointer may be NULL.  blocks (cap entries) is
+ * written for requests that hold blocks; host_image is a borrowed pointer into
+ * the arena, valid while the request stays in HOST; arena_offset is its offset.
+ */
+kvr_status kvr_request_info(kvr_pool *pool, uint64_t req, int32_t *state, int64_t *n_tokens, int32_t *nb,
+                            int32_t *blocks, int32_t cap, const void **host_image, uint64_t *image_bytes,
+                            uint64_t *arena_offset);
+/*
+ * Time the last move of a request took: host_ms from call entry until its work
+ * was enqueued, device_ms from the first enqueued work of that call until this
+ * request's last byte landed.  KVR_ERR_BAD_STATE if it never moved or the move
+ * is still in flight.
+ */
+kvr_status kvr_request_latency(kvr_pool *pool, uint64_t req, double *host_ms, double *device_ms);
+
+/*
+ * Wait until the moves of one request (or KVR_ALL) are complete; polls, never
+ * blocks longer than timeout_ms (< 0 = 60 s): KVR_ERR_TIMEOUT.  Surfaces a
+ * device-side mover error (a bounded wait that ran out) as KVR_ERR_CUDA.
+ */
+kvr_status kvr_wait(kvr_pool *pool, uint64_t req_or_all, int64_t timeout_ms);
+
+kvr_status kvr_pool_stats(kvr_pool *pool, kvr_stats *out);
+/* copies the free queue, head first, into out (cap entries, may be NULL); returns its length */
+int64_t kvr_free_queue(kvr_pool *pool, int32_t *out, int64_t cap);
+/* the DEVICE pool pointer and the HOST arena pointer in use (caller's or the library's) */
+void *kvr_pool_device_ptr(kvr_pool *pool);
+void *kvr_pool_host_arena(kvr_pool *pool);
+/* message of the last error on this thread ("" if none) */
+const char *kvr_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

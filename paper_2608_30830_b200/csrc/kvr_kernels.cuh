@@ -1,0 +1,49 @@
+// Device-side descriptors and launchers of the gather / scatter movers.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+
+namespace kvr {
+
+// One request's share of one launch.  Tiles of a request are numbered
+// q = plane * nb + b (plane = 2*layer + kv, b = logical block), which is also
+// the order of their bytes in the image, so a run of tile ids is one
+// contiguous byte range of the image.
+struct Seg {
+  const int32_t *bt;     // DEVICE: the request's block table (nb entries)
+  char *img;             // address of image byte 0 in the linear buffer this launch reads or writes
+                         // (may lie before the buffer when the launch covers a later part of the image)
+  long long n_tokens;
+  long long tile_begin;  // first tile id of this request handled by the launch
+  long long tile_count;
+  int nb;
+  int pad;
+};
+
+constexpr int kMaxSegs = 1024;   // segments per launch (the host splits larger batches)
+
+struct MoveArgs {
+  const Seg *segs;       // DEVICE
+  int nsegs;
+  long long total_tiles; // sum of tile_count
+  char *pool;            // DEVICE: paged pool base
+  long long plane_stride;// bytes of one (layer, plane): num_blocks * tile_bytes
+  int tile_bytes;        // block_size * row_bytes
+  int row_bytes;         // kv_heads * head_dim * dtype_bytes (multiple of 16)
+  int block_size;
+  int *status;           // DEVICE: error word (0 = fine), written only when a bounded wait runs out
+};
+
+struct BulkShape {       // tuning of the bulk mover
+  int warps;             // independent pipelines per CTA
+  int stages;            // shared-memory stages per pipeline
+  int piece_bytes;       // bytes per bulk copy (multiple of 16, <= tile_bytes rounded)
+};
+
+// gather = pool -> linear, scatter = linear -> pool.  grid_limit caps the number of CTAs (0 = default).
+cudaError_t launch_move_warp(bool gather, const MoveArgs &a, int grid_limit, int sm_count, cudaStream_t s);
+cudaError_t launch_move_bulk(bool gather, const MoveArgs &a, const BulkShape &shape, int grid_limit,
+                             int sm_count, cudaStream_t s);
+cudaError_t bulk_configure(const BulkShape &shape);   // once per device: opt in to large dynamic shared memory
+
+}  // namespace kvr

@@ -1,0 +1,287 @@
+"""ctypes binding of libkvr.so: same names as the C ABI (include/kvr.h), argument marshalling only."""
+import ctypes as C
+import os
+
+import numpy as np
+
+from . import build as _build
+
+OK, RESIDENT, RECOMPUTE, HOST_FULL, HBM_FULL = 0, 1, 2, 3, 4
+ERR_INVALID_ARG, ERR_UNKNOWN_REQUEST, ERR_BAD_STATE, ERR_GEOMETRY = -1, -2, -3, -4
+ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM = -5, -6, -7
+ACTIVE, RETAINED, SUSPENDING, HOST, RESUMING, EXPIRED = 0, 1, 2, 3, 4, 5
+SYNC = 1
+METADATA_ONLY, PROFILE = 1, 2
+ROUTE_STAGED, ROUTE_MAPPED = 1, 2
+KERNEL_WARP, KERNEL_BULK = 1, 2
+ALL = 2**64 - 1
+
+
+class KvrError(RuntimeError):
+    def __init__(self, status, msg):
+        super().__init__("kvr status %d: %s" % (status, msg))
+        self.status = status
+
+
+class Geometry(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("layers", "kv_heads", "head_dim", "dtype_bytes", "block_size")]
+
+
+class Config(C.Structure):
+    _fields_ = [("g", Geometry), ("num_blocks", C.c_int32), ("device", C.c_int32),
+                ("host_capacity_bytes", C.c_uint64), ("chunk_bytes", C.c_uint64),
+                ("staging_slots", C.c_int32), ("route", C.c_int32), ("kernel", C.c_int32),
+                ("max_ctas", C.c_int32), ("flags", C.c_uint32), ("reserved", C.c_uint32),
+                ("device_pool", C.c_void_p), ("host_arena", C.c_void_p),
+                ("initial_free_order", C.POINTER(C.c_int32))]
+
+
+class Stats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("blocks_total", "blocks_free", "blocks_active", "blocks_pinned")] + \
+               [(n, C.c_uint64) for n in ("host_capacity", "host_used", "host_largest_hole")] + \
+               [(n, C.c_int64) for n in ("n_active", "n_retained", "n_host", "n_expired",
+                                         "suspends", "resumes", "resident_resumes", "expires",
+                                         "recompute_marked", "host_full_rejects", "hbm_full_rejects")] + \
+               [(n, C.c_uint64) for n in ("bytes_suspended", "bytes_resumed", "bytes_expired_from_host")] + \
+               [(n, C.c_int64) for n in ("ops_in_flight", "gather_launches", "scatter_launches",
+                                         "d2h_copies", "h2d_copies")] + \
+               [(n, C.c_uint64) for n in ("gather_bytes", "scatter_bytes", "d2h_bytes", "h2d_bytes", "desc_bytes")] + \
+               [(n, C.c_double) for n in ("gather_ms", "scatter_ms")]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+EXPORTS = [
+    "kvr_bytes_per_token", "kvr_pool_create", "kvr_pool_destroy", "kvr_request_admit", "kvr_request_release",
+    "kvr_retain_in_hbm", "kvr_suspend_to_host", "kvr_expire", "kvr_resume_from_host",
+    "kvr_resume_from_host_into", "kvr_export_to_device", "kvr_import_from_device", "kvr_request_info",
+    "kvr_request_latency", "kvr_wait", "kvr_pool_stats", "kvr_free_queue", "kvr_pool_device_ptr",
+    "kvr_pool_host_arena", "kvr_last_error",
+]
+
+_lib = None
+
+
+def lib():
+    """Load libkvr.so (building it with nvcc if the sources are newer).  Raises if that fails."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    try:
+        path = _build.build()
+    except Exception as e:  # no silent fallback: the CUDA library is the product
+        if not os.path.exists(_build.SO):
+            raise ImportError("libkvr.so is missing and could not be built: %r" % (e,))
+        path = _build.SO
+    L = C.CDLL(path)
+    i32, i64, u32, u64, vp = C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_void_p
+    pi32, pu64 = C.POINTER(C.c_int32), C.POINTER(C.c_uint64)
+    L.kvr_bytes_per_token.restype = u64
+    L.kvr_bytes_per_token.argtypes = [C.POINTER(Geometry)]
+    L.kvr_pool_create.restype = i32
+    L.kvr_pool_create.argtypes = [C.POINTER(Config), C.POINTER(vp)]
+    L.kvr_pool_destroy.restype = i32
+    L.kvr_pool_destroy.argtypes = [vp]
+    L.kvr_request_admit.restype = i32
+    L.kvr_request_admit.argtypes = [vp, u64, i64, pi32, i32]
+    L.kvr_request_release.restype = i32
+    L.kvr_request_release.argtypes = [vp, u64]
+    for name in ("kvr_retain_in_hbm", "kvr_expire"):
+        f = getattr(L, name)
+        f.restype = i32
+        f.argtypes = [vp, pu64, i32, pi32]
+    for name in ("kvr_suspend_to_host", "kvr_resume_from_host"):
+        f = getattr(L, name)
+        f.restype = i32
+        f.argtypes = [vp, pu64, i32, u32, pi32]
+    L.kvr_resume_from_host_into.restype = i32
+    L.kvr_resume_from_host_into.argtypes = [vp, u64, pi32, i32, u32]
+    for name in ("kvr_export_to_device", "kvr_import_from_device"):
+        f = getattr(L, name)
+        f.restype = i32
+        f.argtypes = [vp, pu64, i32, vp, u64, pu64, u32]
+    L.kvr_request_info.restype = i32
+    L.kvr_request_info.argtypes = [vp, u64, pi32, C.POINTER(i64), pi32, pi32, i32, C.POINTER(vp), pu64, pu64]
+    L.kvr_request_latency.restype = i32
+    L.kvr_request_latency.argtypes = [vp, u64, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    L.kvr_wait.restype = i32
+    L.kvr_wait.argtypes = [vp, u64, i64]
+    L.kvr_pool_stats.restype = i32
+    L.kvr_pool_stats.argtypes = [vp, C.POINTER(Stats)]
+    L.kvr_free_queue.restype = i64
+    L.kvr_free_queue.argtypes = [vp, pi32, i64]
+    L.kvr_pool_device_ptr.restype = vp
+    L.kvr_pool_device_ptr.argtypes = [vp]
+    L.kvr_pool_host_arena.restype = vp
+    L.kvr_pool_host_arena.argtypes = [vp]
+    L.kvr_last_error.restype = C.c_char_p
+    L.kvr_last_error.argtypes = []
+    _lib = L
+    return L
+
+
+def last_error():
+    return lib().kvr_last_error().decode()
+
+
+def bytes_per_token(layers, kv_heads, head_dim, dtype_bytes, block_size=16):
+    g = Geometry(layers, kv_heads, head_dim, dtype_bytes, block_size)
+    return int(lib().kvr_bytes_per_token(C.byref(g)))
+
+
+def _i32p(a):
+    return a.ctypes.data_as(C.POINTER(C.c_int32))
+
+
+def _u64p(a):
+    return a.ctypes.data_as(C.POINTER(C.c_uint64))
+
+
+class Pool:
+    """kvr_pool handle.  Methods are the C calls with numpy / int marshalling; statuses are returned, not raised,
+    except for errors of pool creation."""
+
+    def __init__(self, layers, kv_heads, head_dim, dtype_bytes, block_size, num_blocks, host_capacity_bytes,
+                 initial_free_order=None, device=0, chunk_bytes=0, staging_slots=0, route=0, kernel=0,
+                 max_ctas=0, flags=0, device_pool=None, host_arena=None):
+        self.geom = (layers, kv_heads, head_dim, dtype_bytes, block_size)
+        self.NB = num_blocks
+        cfg = Config()
+        cfg.g = Geometry(*self.geom)
+        cfg.num_blocks, cfg.device = num_blocks, device
+        cfg.host_capacity_bytes, cfg.chunk_bytes, cfg.staging_slots = host_capacity_bytes, chunk_bytes, staging_slots
+        cfg.route, cfg.kernel, cfg.max_ctas, cfg.flags = route, kernel, max_ctas, flags
+        cfg.device_pool = device_pool
+        cfg.host_arena = host_arena
+        order = None
+        if initial_free_order is not None:
+            order = np.ascontiguousarray(initial_free_order, dtype=np.int32)
+            if order.size != num_blocks:
+                raise ValueError("initial_free_order must have num_blocks entries")
+            cfg.initial_free_order = _i32p(order)
+        h = C.c_void_p()
+        st = lib().kvr_pool_create(C.byref(cfg), C.byref(h))
+        if st != OK:
+            raise KvrError(st, last_error())
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            st = lib().kvr_pool_destroy(self._h)
+            self._h = None
+            return st
+        return OK
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+    # -- lifecycle
+    def admit(self, rid, n_tokens):
+        nb = max(0, -(-n_tokens // self.geom[4]))
+        out = np.zeros(max(nb, 1), dtype=np.int32)
+        st = lib().kvr_request_admit(self._h, rid, n_tokens, _i32p(out), nb)
+        return st, (out[:nb].copy() if st == OK else None)
+
+    def release(self, rid):
+        return lib().kvr_request_release(self._h, rid)
+
+    # -- the named calls
+    def _batch(self, fn, ids, *flags):
+        ids = np.ascontiguousarray(ids, dtype=np.uint64)
+        per = np.zeros(max(len(ids), 1), dtype=np.int32)
+        st = fn(self._h, _u64p(ids), len(ids), *flags, _i32p(per))
+        return st, per[:len(ids)].tolist()
+
+    def retain_in_hbm(self, ids):
+        return self._batch(lib().kvr_retain_in_hbm, ids)
+
+    def suspend_to_host(self, ids, flags=0):
+        return self._batch(lib().kvr_suspend_to_host, ids, flags)
+
+    def expire(self, ids):
+        return self._batch(lib().kvr_expire, ids)
+
+    def resume_from_host(self, ids, flags=0):
+        return self._batch(lib().kvr_resume_from_host, ids, flags)
+
+    def resume_from_host_into(self, rid, blocks, flags=0):
+        blocks = np.ascontiguousarray(blocks, dtype=np.int32)
+        return lib().kvr_resume_from_host_into(self._h, rid, _i32p(blocks), len(blocks), flags)
+
+    def _device_copy(self, fn, ids, ptr, capacity, flags):
+        ids = np.ascontiguousarray(ids, dtype=np.uint64)
+        offs = np.zeros(max(len(ids), 1), dtype=np.uint64)
+        st = fn(self._h, _u64p(ids), len(ids), ptr, capacity, _u64p(offs), flags)
+        return st, offs[:len(ids)].copy()
+
+    def export_to_device(self, ids, device_ptr, capacity, flags=0):
+        return self._device_copy(lib().kvr_export_to_device, ids, device_ptr, capacity, flags)
+
+    def import_from_device(self, ids, device_ptr, capacity, flags=0):
+        return self._device_copy(lib().kvr_import_from_device, ids, device_ptr, capacity, flags)
+
+    # -- observation
+    def info(self, rid):
+        state, n, nb = C.c_int32(), C.c_int64(), C.c_int32()
+        img, nbytes, off = C.c_void_p(), C.c_uint64(), C.c_uint64()
+        st = lib().kvr_request_info(self._h, rid, C.byref(state), C.byref(n), C.byref(nb), None, 0,
+                                    C.byref(img), C.byref(nbytes), C.byref(off))
+        if st != OK:
+            return st, None
+        d = dict(state=state.value, n_tokens=n.value, nb=nb.value, image_bytes=nbytes.value,
+                 arena_offset=off.value, blocks=None, image_ptr=img.value)
+        if nb.value >= 0:
+            blocks = np.zeros(max(nb.value, 1), dtype=np.int32)
+            st2 = lib().kvr_request_info(self._h, rid, None, None, None, _i32p(blocks), nb.value, None, None, None)
+            if st2 == OK and state.value in (ACTIVE, RETAINED, RESUMING):
+                d["blocks"] = blocks[:nb.value].copy()
+        return st, d
+
+    def host_image(self, rid):
+        """Borrowed uint8 numpy view of a HOST request's image in the pinned arena (wait for the suspend first)."""
+        st, d = self.info(rid)
+        if st != OK or not d["image_ptr"]:
+            return None
+        if d["image_bytes"] == 0:
+            return np.zeros(0, dtype=np.uint8)
+        buf = (C.c_uint8 * d["image_bytes"]).from_address(d["image_ptr"])
+        return np.frombuffer(buf, dtype=np.uint8)
+
+    def latency(self, rid):
+        h, dv = C.c_double(), C.c_double()
+        st = lib().kvr_request_latency(self._h, rid, C.byref(h), C.byref(dv))
+        return st, h.value, dv.value
+
+    def wait(self, rid=ALL, timeout_ms=-1):
+        return lib().kvr_wait(self._h, rid, timeout_ms)
+
+    def stats(self):
+        s = Stats()
+        st = lib().kvr_pool_stats(self._h, C.byref(s))
+        if st != OK:
+            raise KvrError(st, last_error())
+        return s.as_dict()
+
+    def free_queue(self):
+        n = int(lib().kvr_free_queue(self._h, None, 0))
+        out = np.zeros(max(n, 1), dtype=np.int32)
+        lib().kvr_free_queue(self._h, _i32p(out), n)
+        return out[:n].copy()
+
+    @property
+    def device_ptr(self):
+        return lib().kvr_pool_device_ptr(self._h)
+
+    @property
+    def host_arena_ptr(self):
+        return lib().kvr_pool_host_arena(self._h)

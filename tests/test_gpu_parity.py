@@ -1,0 +1,218 @@
+"""GPU parity: the CUDA library against the CPU oracle, byte for byte, through the C ABI.
+
+Small cases compare every host image and the whole pool; they span several tiles, ragged tails, empty
+requests, chunk boundaries that cut requests, more requests than one launch holds, both routes and both
+kernels, and un-synchronised call sequences whose hazards the library must order itself."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from common import check_invariants, random_script, run_script
+from kvr_synth import CONFIGS, context_lengths, free_order
+from paper_2608_30830_b200 import kvr
+
+pytestmark = [pytest.mark.gpu, pytest.mark.skipif(not torch.cuda.is_available(), reason="needs a CUDA device")]
+
+from gpu_common import Twin  # noqa: E402
+
+MODES = [
+    pytest.param(dict(route=kvr.ROUTE_STAGED, kernel=kvr.KERNEL_WARP), id="staged-warp"),
+    pytest.param(dict(route=kvr.ROUTE_STAGED, kernel=kvr.KERNEL_BULK), id="staged-bulk"),
+    pytest.param(dict(route=kvr.ROUTE_MAPPED, kernel=kvr.KERNEL_WARP), id="mapped-warp"),
+    pytest.param(dict(route=kvr.ROUTE_MAPPED, kernel=kvr.KERNEL_BULK), id="mapped-bulk"),
+]
+SMALL = (3, 2, 16, 2, 8)          # L, H, D, e, BS: 64-byte rows, 512-byte tiles, 384 bytes per token
+LENGTHS = [0, 1, 7, 8, 9, 64, 67, 200, 3, 16]
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_suspend_then_resume_small(mode):
+    t = Twin(SMALL, 128, 1 << 22, seed=1, chunk_bytes=4096, staging_slots=2, **mode)
+    ids = list(range(len(LENGTHS)))
+    for rid, n in zip(ids, LENGTHS):
+        a, b = t.both("admit", rid, n)
+        assert a[0] == b[0] == orc.OK and a[1].tolist() == b[1].tolist()
+    a, b = t.both("suspend_to_host", ids)
+    assert a == b
+    t.assert_same_images(ids)
+    t.assert_same_pool()                                  # a suspend does not touch the pool
+    a, b = t.both("resume_from_host", ids)
+    assert a == b
+    for rid in ids:
+        assert t.o.info(rid)[1]["blocks"].tolist() == t.g.info(rid)[1]["blocks"].tolist()
+    t.assert_same_pool()                                  # only valid slots of the new blocks changed
+    check_invariants(t.g, ids)
+    s = t.g.stats()
+    assert s["gather_launches"] >= 1 and s["scatter_launches"] >= 1
+    assert s["gather_bytes"] == s["scatter_bytes"] == sum(LENGTHS) * 384
+    t.close()
+
+
+@pytest.mark.parametrize("mode", MODES[:2])
+def test_export_import_kernels_alone(mode):
+    """gather and scatter kernels HBM to HBM, against the oracle's per-element loops."""
+    t = Twin(SMALL, 96, 0, seed=2, **mode)
+    L, H, D, e, BS = SMALL
+    ids = list(range(len(LENGTHS)))
+    tables = {}
+    for rid, n in zip(ids, LENGTHS):
+        tables[rid] = t.g.admit(rid, n)[1]
+        t.o.admit(rid, n)
+    cap = sum(-(-n * 384 // 256) * 256 for n in LENGTHS) + 256
+    buf = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+    st, offs = t.g.export_to_device(ids, buf.data_ptr(), cap, kvr.SYNC)
+    assert st == kvr.OK, kvr.last_error()
+    host = buf.cpu().numpy()
+    for rid, n, off in zip(ids, LENGTHS, offs):
+        want = orc.gather(t.o.data, L, H, D, e, BS, t.NB, tables[rid], n)
+        assert off % 256 == 0 and np.array_equal(host[int(off):int(off) + want.size], want)
+    # scatter new content back through the same tables
+    new = np.random.default_rng(5).integers(0, 256, size=cap, dtype=np.uint8)
+    buf.copy_(torch.from_numpy(new))
+    torch.cuda.synchronize()
+    st, offs2 = t.g.import_from_device(ids, buf.data_ptr(), cap, kvr.SYNC)
+    assert st == kvr.OK and offs2.tolist() == offs.tolist()
+    for rid, n, off in zip(ids, LENGTHS, offs):
+        orc.scatter(t.o.data, new[int(off):int(off) + n * 384], L, H, D, e, BS, t.NB, tables[rid], n)
+    t.assert_same_pool()
+    assert t.g.export_to_device(ids, buf.data_ptr(), 100)[0] == kvr.ERR_INVALID_ARG
+    t.close()
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_random_scripts_with_data(mode, seed):
+    """Seeded call scripts (legal and illegal calls, HOST_FULL, HBM_FULL, relabelling) with no waits between
+    calls: statuses, tables, offsets, every host image at the end and the final pool must equal the oracle's."""
+    NB, cap = 48, 10 * 4096
+    t = Twin(SMALL, NB, cap, seed=seed, chunk_bytes=4096, staging_slots=2, **mode)
+    ops = random_script(100 + seed, 300, max_tokens=70)
+    la = run_script(t.o, ops)
+    lb = run_script(t.g, ops)
+    for (op, sa, pa, snap_a), (_, sb, pb, snap_b) in zip(la, lb):
+        assert (sa, pa) == (sb, pb) and snap_a == snap_b, op
+    t.assert_same_images(range(12))
+    t.assert_same_pool()
+    check_invariants(t.g, range(12))
+    t.close()
+
+
+@pytest.mark.parametrize("mode", MODES[:2])
+def test_images_checked_after_every_move(mode):
+    NB, cap = 48, 12 * 4096
+    t = Twin(SMALL, NB, cap, seed=7, chunk_bytes=8192, staging_slots=3, **mode)
+    ops = random_script(7, 120, max_tokens=70)
+
+    def after(op, st):
+        if op[0] in ("suspend", "resume", "resume_into"):
+            t.assert_same_images(range(12))
+    # run the oracle one call ahead of the library so images can be compared after each library call
+    lo = []
+    for op in ops:
+        lo += run_script(t.o, [op])
+        lg = run_script(t.g, [op], after_each=after)
+        assert lo[-1][1:] == lg[-1][1:], op
+    t.assert_same_pool()
+    t.close()
+
+
+@pytest.mark.parametrize("kernel", [kvr.KERNEL_WARP, kvr.KERNEL_BULK])
+def test_more_requests_than_one_launch_holds(kernel):
+    geom = (1, 1, 16, 1, 2)                                # 16-byte rows, 32-byte tiles
+    n_req = 1100 * 2 + 7
+    t = Twin(geom, 8192, 1 << 24, seed=3, kernel=kernel, chunk_bytes=1 << 20)
+    rng = np.random.default_rng(3)
+    ids = list(range(n_req))
+    for rid in ids:
+        n = int(rng.integers(0, 6))
+        assert t.both("admit", rid, n)[1][0] == kvr.OK
+    a, b = t.both("suspend_to_host", ids)
+    assert a == b
+    t.assert_same_images(ids)
+    a, b = t.both("resume_from_host", ids)
+    assert a == b
+    t.assert_same_pool()
+    t.close()
+
+
+def test_hazards_without_waiting():
+    """Blocks freed by a suspend are taken by the next resume, host ranges freed by a resume are taken by the
+    next suspend, the same request is moved again while its last move is in flight: no wait in between."""
+    geom = (4, 2, 64, 2, 16)                               # 256-byte rows, 4 KiB tiles, 2 KiB per token
+    NB = 64
+    t = Twin(geom, NB, 3 << 20, seed=9, chunk_bytes=16384, staging_slots=2)
+    lens = [300, 257, 131, 16]                             # 19 + 17 + 9 + 1 = 46 of 64 blocks
+    for rid, n in enumerate(lens):
+        assert t.both("admit", rid, n)[1][0] == kvr.OK
+    for rnd in range(6):
+        a, b = t.both("suspend_to_host", [0, 1])
+        assert a == b
+        a, b = t.both("resume_from_host", [1, 0])          # takes blocks the suspend just released
+        assert a == b
+        a, b = t.both("suspend_to_host", [2, 3, 0])        # request 0 again, its resume still in flight
+        assert a == b
+        a, b = t.both("resume_from_host", [0, 2, 3])
+        assert a == b
+    for rid in range(4):
+        assert t.o.info(rid)[1]["blocks"].tolist() == t.g.info(rid)[1]["blocks"].tolist()
+    t.assert_same_pool()
+    t.close()
+
+
+def test_transient_states_and_latency():
+    geom = (4, 2, 64, 2, 16)
+    t = Twin(geom, 64, 1 << 21, seed=4)
+    t.both("admit", 1, 200)
+    assert t.g.latency(1)[0] == kvr.ERR_BAD_STATE
+    t.g.suspend_to_host([1])
+    t.o.suspend_to_host([1])
+    st = t.g.info(1)[1]["state"]
+    assert st in (kvr.SUSPENDING, kvr.HOST)
+    assert t.g.wait(1) == kvr.OK and t.g.info(1)[1]["state"] == kvr.HOST
+    st, host_ms, dev_ms = t.g.latency(1)
+    assert st == kvr.OK and host_ms > 0 and dev_ms > 0
+    t.g.resume_from_host([1], kvr.SYNC)
+    t.o.resume_from_host([1])
+    assert t.g.info(1)[1]["state"] == kvr.ACTIVE
+    assert t.g.wait(99) == kvr.ERR_UNKNOWN_REQUEST
+    t.assert_same_pool()
+    t.close()
+
+
+def test_caller_owned_pinned_arena_and_grid_cap():
+    geom = (4, 2, 64, 2, 16)
+    cap = 1 << 21
+    arena = torch.empty(cap + 4096, dtype=torch.uint8).pin_memory()
+    base = (arena.data_ptr() + 4095) // 4096 * 4096
+    t = Twin(geom, 64, cap, seed=6, host_arena=base, max_ctas=3, chunk_bytes=65536)
+    t.both("admit", 1, 500)
+    t.both("admit", 2, 123)
+    assert t.both("suspend_to_host", [1, 2])[1][0] == kvr.OK
+    t.assert_same_images([1, 2])
+    assert t.g.host_arena_ptr == base
+    t.both("resume_from_host", [2, 1])
+    t.assert_same_pool()
+    t.close()
+
+
+def test_tiny_config_full_size():
+    """The benchmark's smallest configuration at full size: whole pool and every image compared."""
+    w = CONFIGS["tiny"]
+    seed = 20260830
+    order = free_order(seed, w.num_blocks)
+    lens = context_lengths(w.length_rule, w.n_requests, seed)
+    t = Twin(w.geom, w.num_blocks, 1 << 28, seed=seed, order=order, flags=kvr.PROFILE)
+    ids = list(range(w.n_requests))
+    for rid, n in zip(ids, lens):
+        assert t.both("admit", rid, int(n))[1][0] == kvr.OK
+    a, b = t.both("suspend_to_host", ids)
+    assert a == b == (kvr.OK, [kvr.OK] * 4)
+    t.assert_same_images(ids)
+    a, b = t.both("resume_from_host", ids)
+    assert a == b
+    t.assert_same_pool()
+    s = t.g.stats()
+    assert s["bytes_suspended"] == s["bytes_resumed"] == int(lens.sum()) * 32768
+    assert s["gather_ms"] > 0 and s["scatter_ms"] > 0
+    t.close()
