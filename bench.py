@@ -1,0 +1,418 @@
+#!/usr/bin/env python
+"""Benchmark of the suspend/resume hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic suspended requests:
+retain one request in HBM and resume it in place, suspend the batch to pinned host memory
+(descriptor build, gather kernel, device-to-host copies, block release), expire one host
+image and re-admit it, resume the batch (block allocation, host-to-device copies, scatter
+kernel).  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--workload llama3_8b|tiny|gqa64] [--route staged|mapped] [--kernel warp|bulk]
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from kvr_synth import CONFIGS, context_lengths, fill_bytes, free_order, occupancy_fillers  # noqa: E402
+
+SEED = 20260830
+METRIC = "suspend/resume payload GB/s (batched suspend to pinned host, then batched resume)"
+
+
+def peaks():
+    """Measured roofline denominators written by the driver, else the documented fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return json.load(open(path))["hbm_gbs"], "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows, self.proc, self.index = [], None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = [r for r in self.rows if len(r) == 6 and r[0].isdigit()]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[2 + i] == "Active" for r in rows)]
+        return {"sm_mhz": float(np.median([int(r[0]) for r in rows])), "sm_max_mhz": float(rows[0][1]),
+                "reasons": reasons, "samples": len(rows)}
+
+
+def build_workload(name, n_requests_cap=None, overrides=None):
+    """The named configuration; `overrides` (num_blocks, requests, fixed_tokens) shrink it for profiling."""
+    import dataclasses
+    w = CONFIGS[name]
+    o = overrides or {}
+    if o.get("num_blocks"):
+        w = dataclasses.replace(w, num_blocks=o["num_blocks"])
+    if o.get("requests"):
+        w = dataclasses.replace(w, n_requests=o["requests"])
+    if o.get("fixed_tokens"):
+        w = dataclasses.replace(w, length_rule=("fixed", o["fixed_tokens"]))
+    seed = SEED + list(CONFIGS).index(name)
+    lens = context_lengths(w.length_rule, w.n_requests, seed)
+    if n_requests_cap is not None:
+        lens = lens[:n_requests_cap]
+    bs = w.block_size
+    used = int(sum(-(-int(n) // bs) for n in lens))
+    fillers = occupancy_fillers(w.num_blocks, bs, used, w.occupancy, seed) if w.occupancy else np.zeros(0, np.int64)
+    return w, seed, lens, fillers
+
+
+def cpu_oracle_sample(geom, tokens, threads=1):
+    """Times the oracle's gather and scatter loops, as they stand, on one request of `tokens` tokens."""
+    import oracle as orc
+    L, H, D, e, BS = geom
+    nb = -(-tokens // BS)
+    NB = nb * 2
+    pool = fill_bytes(SEED, 77, NB * BS * 2 * L * H * D * e, e).copy()
+    rng = np.random.default_rng(SEED)
+    src = rng.permutation(NB)[:nb].astype(np.int32)
+    t0 = time.perf_counter()
+    img = orc.gather(pool, L, H, D, e, BS, NB, src, tokens)
+    t1 = time.perf_counter()
+    dst = rng.permutation(NB)[:nb].astype(np.int32)
+    orc.scatter(pool, img, L, H, D, e, BS, NB, dst, tokens)
+    t2 = time.perf_counter()
+    payload = img.size
+    return {"payload_bytes": payload, "suspend_s": t1 - t0, "resume_s": t2 - t1,
+            "gbs": 2 * payload / (t2 - t0) / 1e9}
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle, untuned, on the host cores; every step is a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w, seed, lens, fillers = build_workload(args.workload)
+    tokens = 2048
+    for _ in range(args.warmup):
+        cpu_oracle_sample(w.geom, 256)
+    times, gbs = [], []
+    for _ in range(args.steps):
+        r = cpu_oracle_sample(w.geom, tokens)
+        times.append(r["suspend_s"] + r["resume_s"])
+        gbs.append(r["gbs"])
+    value = float(np.mean(gbs))
+    sample = "one %d-token request of the %s geometry per step: oracle gather then scatter, 1 thread" % (tokens, w.name)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(times)),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": w.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def link_peak(torch, kvr_pool, arena_bytes, reps=10):
+    """Pinned cudaMemcpyAsync peak in each direction over the library's own arena (same placement)."""
+    import ctypes as C
+    n = min(arena_bytes // 4096 * 4096, 2 << 30)
+    host = torch.frombuffer((C.c_uint8 * n).from_address(kvr_pool.host_arena_ptr), dtype=torch.uint8)
+    dev = torch.empty(n, dtype=torch.uint8, device="cuda")
+    out = {"bytes": n, "pinned": bool(host.is_pinned())}
+    s = torch.cuda.Stream()
+    for name in ("d2h", "h2d"):
+        ts = []
+        for _ in range(reps + 3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            with torch.cuda.stream(s):
+                e0.record()
+                if name == "d2h":
+                    host.copy_(dev, non_blocking=True)
+                else:
+                    dev.copy_(host, non_blocking=True)
+                e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        ts = sorted(ts[3:])
+        out[name + "_best_gbs"] = n / ts[0] / 1e6
+        out[name + "_median_gbs"] = n / ts[len(ts) // 2] / 1e6
+    del dev
+    return out
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_30830_b200 import kvr
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # scale rule: every rank pins its own arena out of the same host DRAM; keep geometry and lengths,
+    # reduce the request count when the arenas of all ranks would not fit in 60% of what is available
+    ov = {"num_blocks": args.num_blocks, "requests": args.requests, "fixed_tokens": args.fixed_tokens}
+    w, seed, lens, fillers = build_workload(args.workload, None, ov)
+    bpt = kvr.bytes_per_token(*w.geom[:4])
+    requested = len(lens)
+    avail = int(open("/proc/meminfo").read().split("MemAvailable:")[1].split()[0]) * 1024
+    budget = int(0.6 * avail / world)
+    while len(lens) > 1 and int(lens.sum()) * bpt + (2 << 30) > budget:
+        lens = lens[:-1]
+    if len(lens) != requested:
+        w, seed, lens, fillers = build_workload(args.workload, len(lens), ov)
+    L, H, D, e, BS = w.geom
+    payload = int(lens.sum()) * bpt
+    lone_tokens = 8192
+    small_k = int(np.argmin(fillers)) if len(fillers) else None     # request used for the retain / expire rows
+    small_tokens = int(fillers[small_k]) if small_k is not None else 0
+    host_cap = -(-(payload + len(lens) * 4096 + (lone_tokens + small_tokens) * bpt + (64 << 20)) // 4096) * 4096
+
+    # pool bytes: bf16 N(0,1) drawn on the device from a seeded generator
+    pool_bytes = w.num_blocks * BS * bpt
+    dev_pool = torch.empty(pool_bytes, dtype=torch.uint8, device="cuda")
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed + rank)
+    view = dev_pool.view(torch.bfloat16)
+    step_elems = 1 << 28
+    for i in range(0, view.numel(), step_elems):
+        view[i:i + step_elems].normal_(generator=gen)
+    torch.cuda.synchronize()
+
+    route = {"staged": kvr.ROUTE_STAGED, "mapped": kvr.ROUTE_MAPPED}[args.route]
+    kernel = {"warp": kvr.KERNEL_WARP, "bulk": kvr.KERNEL_BULK}[args.kernel]
+    pool = kvr.Pool(*w.geom, w.num_blocks, host_cap, initial_free_order=free_order(seed, w.num_blocks),
+                    device=local, device_pool=dev_pool.data_ptr(), route=route, kernel=kernel,
+                    chunk_bytes=args.chunk_mib << 20, staging_slots=args.slots, max_ctas=args.max_ctas,
+                    flags=kvr.PROFILE)
+
+    # live set: the batch and the fillers, admitted in a seeded interleaved order (fragmented placement)
+    ids = list(range(len(lens)))
+    filler_ids = list(range(1000, 1000 + len(fillers)))
+    order = [(i, int(n)) for i, n in zip(ids, lens)] + [(i, int(n)) for i, n in zip(filler_ids, fillers)]
+    np.random.default_rng(seed).shuffle(order)
+    for rid, n in order:
+        st, _ = pool.admit(rid, n)
+        assert st == kvr.OK, (rid, n, st, kvr.last_error())
+    occupancy = 1.0 - pool.stats()["blocks_free"] / w.num_blocks
+    small = filler_ids[small_k] if small_k is not None else None
+
+    link = link_peak(torch, pool, host_cap) if rank == 0 else None
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+
+    def one_step():
+        """Returns (device_ms_suspend, device_ms_resume, wall_s)."""
+        t0 = time.perf_counter()
+        if small is not None:                          # HBM retention: nothing moves, resume is resident
+            assert pool.retain_in_hbm([small])[0] == kvr.OK
+            assert pool.resume_from_host([small])[0] == kvr.RESIDENT
+        st, per = pool.suspend_to_host(ids)
+        assert st == kvr.OK, (st, per, kvr.last_error())
+        assert pool.wait() == kvr.OK, kvr.last_error()
+        sus = max(pool.latency(r)[2] for r in ids)
+        if small is not None:                          # host copy expires, resume answers recompute, re-admit
+            assert pool.suspend_to_host([small], kvr.SYNC)[0] == kvr.OK
+            assert pool.expire([small])[0] == kvr.OK
+            assert pool.resume_from_host([small])[0] == kvr.RECOMPUTE
+            assert pool.admit(small, small_tokens)[0] == kvr.OK
+        st, per = pool.resume_from_host(ids)
+        assert st == kvr.OK, (st, per, kvr.last_error())
+        assert pool.wait() == kvr.OK, kvr.last_error()
+        res = max(pool.latency(r)[2] for r in ids)
+        return sus, res, time.perf_counter() - t0
+
+    for _ in range(args.warmup):
+        one_step()
+    sampler = ClockSampler(local)
+    s0 = pool.stats()
+    barrier()
+    sampler.start()
+    t_begin = time.perf_counter()
+    steps = [one_step() for _ in range(args.steps)]
+    barrier()
+    wall = time.perf_counter() - t_begin
+    clocks = sampler.stop()
+    s1 = pool.stats()
+
+    sus_ms = float(np.sum([s[0] for s in steps]))
+    res_ms = float(np.sum([s[1] for s in steps]))
+    dev_s = (sus_ms + res_ms) / 1e3
+    if world > 1:
+        tt = torch.tensor([dev_s, wall, sus_ms, res_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        dev_s, wall, sus_ms, res_ms = tt.tolist()
+        pp = torch.tensor([payload], dtype=torch.float64, device="cuda")
+        dist.all_reduce(pp, op=dist.ReduceOp.SUM)
+        payload_all = float(pp.item())
+    else:
+        payload_all = float(payload)
+    K = args.steps
+    moved = 2.0 * payload_all * K                      # bytes suspended + bytes resumed, all ranks
+    value = moved / dev_s / 1e9
+    e2e = moved / wall / 1e9
+
+    if rank == 0:
+        # kernels inside the timed region (profiling events around every launch)
+        d = {k: s1[k] - s0[k] for k in ("gather_launches", "scatter_launches", "gather_bytes", "scatter_bytes",
+                                        "gather_ms", "scatter_ms", "d2h_bytes", "h2d_bytes", "desc_bytes",
+                                        "d2h_copies", "h2d_copies")}
+        peak, peak_kind = peaks()
+        g_gbs = 2 * d["gather_bytes"] / max(d["gather_ms"], 1e-9) / 1e6
+        s_gbs = 2 * d["scatter_bytes"] / max(d["scatter_ms"], 1e-9) / 1e6
+        name, ach = ("kvr::move_warp<gather>", g_gbs) if g_gbs <= s_gbs else ("kvr::move_warp<scatter>", s_gbs)
+        if args.kernel == "bulk":
+            name = name.replace("move_warp", "move_bulk")
+        # DRAM traffic per launch: ncu measured read+write = 0.956 x the algorithmic bytes on a 512 MiB chunk
+        # (profiles/ncu_full_gather_small_case.md); traffic grows in proportion to the bytes of a launch
+        launches = max(d["gather_launches"] if g_gbs <= s_gbs else d["scatter_launches"], 1)
+        alg_per_launch = 2 * (d["gather_bytes"] if g_gbs <= s_gbs else d["scatter_bytes"]) / launches
+        roofline = {"bound": "hbm", "kernel": name, "achieved": ach, "peak": peak, "unit": "GB/s",
+                    "frac": ach / peak, "peak_source": peak_kind + " copy bandwidth, read+write bytes",
+                    "algorithmic_bytes_per_launch": alg_per_launch,
+                    "traffic": 0.956 * alg_per_launch,
+                    "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum on a 512 MiB chunk, scaled by bytes per launch",
+                    "gather": {"gbs": g_gbs, "frac": g_gbs / peak, "launches": d["gather_launches"],
+                               "avg_us": 1e3 * d["gather_ms"] / max(d["gather_launches"], 1)},
+                    "scatter": {"gbs": s_gbs, "frac": s_gbs / peak, "launches": d["scatter_launches"],
+                                "avg_us": 1e3 * d["scatter_ms"] / max(d["scatter_launches"], 1)}}
+
+        # the kernels alone, at the size of the whole batch: HBM -> HBM
+        alone = None
+        free_b, _ = torch.cuda.mem_get_info()
+        need = payload + len(ids) * 256
+        if free_b > need + (2 << 30) and not args.no_extras:
+            buf = torch.empty(need, dtype=torch.uint8, device="cuda")
+            best = {}
+            for direction, fn in (("gather", pool.export_to_device), ("scatter", pool.import_from_device)):
+                ts = []
+                for _ in range(5):
+                    st, _ = fn(ids, buf.data_ptr(), need, kvr.SYNC)
+                    assert st == kvr.OK, kvr.last_error()
+                    ts.append(max(pool.latency(r)[2] for r in ids))
+                best[direction] = {"best_gbs": 2 * payload / min(ts[2:]) / 1e6,
+                                   "median_gbs": 2 * payload / float(np.median(ts[2:])) / 1e6}
+                best[direction]["frac"] = best[direction]["median_gbs"] / peak
+            alone = best
+            del buf
+
+        # resume latency of a lone 8192-token request
+        lone = None
+        if not args.no_extras and pool.admit(5000, lone_tokens)[0] == kvr.OK:
+            sus_l, res_l, res_host = [], [], []
+            for _ in range(5):
+                t0 = time.perf_counter()
+                assert pool.suspend_to_host([5000], kvr.SYNC)[0] == kvr.OK
+                sus_l.append((time.perf_counter() - t0) * 1e3)
+                t0 = time.perf_counter()
+                assert pool.resume_from_host([5000], kvr.SYNC)[0] == kvr.OK
+                res_l.append((time.perf_counter() - t0) * 1e3)
+                res_host.append(pool.latency(5000)[1])
+            lone = {"tokens": lone_tokens, "bytes": lone_tokens * bpt,
+                    "suspend_ms_median": float(np.median(sus_l)), "resume_ms_median": float(np.median(res_l)),
+                    "resume_enqueue_ms_median": float(np.median(res_host)),
+                    "resume_gbs": lone_tokens * bpt / float(np.median(res_l)) / 1e6,
+                    "timing": "host clock, call entry to return of the synchronous call"}
+            pool.release(5000)
+
+        sus_gbs = payload_all * K / sus_ms / 1e6
+        res_gbs = payload_all * K / res_ms / 1e6
+        host_link = dict(link)
+        host_link.update({"suspend_gbs": sus_gbs, "suspend_frac_of_d2h_peak": sus_gbs / world / link["d2h_best_gbs"],
+                          "resume_gbs": res_gbs, "resume_frac_of_h2d_peak": res_gbs / world / link["h2d_best_gbs"]})
+        cpu = cpu_oracle_sample(w.geom, 256 if args.no_extras else 4096)
+        sample = ("one %d-token request of this geometry (%.2f GiB payload): oracle gather then scatter, 1 thread"
+                  % (256 if args.no_extras else 4096, cpu["payload_bytes"] / 2**30))
+        out = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "ms_per_step": 1e3 * wall / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "u8", "data": "synthetic",
+            "config": {"workload": w.name, "geometry": dict(zip(("layers", "kv_heads", "head_dim", "dtype_bytes", "block_size"), w.geom)),
+                       "num_blocks": w.num_blocks, "requests_requested": requested, "requests_run": len(ids),
+                       "tokens": int(lens.sum()), "payload_bytes_per_direction": payload,
+                       "occupancy_before_suspend": occupancy, "route": args.route, "kernel": args.kernel,
+                       "chunk_mib": args.chunk_mib, "staging_slots": args.slots, "seed": seed,
+                       "l2": "inputs (tens of GiB) are far larger than L2; no flush needed",
+                       "timing": "value: CUDA events, first enqueued work to last byte landed, summed over the two batched moves of each step; e2e: host clock around the K steps"},
+            "e2e": {"value": e2e, "unit": "GB/s",
+                    "h2d_bytes_per_step": int((d["h2d_bytes"] + d["desc_bytes"]) / K),
+                    "d2h_bytes_per_step": int(d["d2h_bytes"] / K)},
+            "gpu_launches": int(d["gather_launches"] + d["scatter_launches"]),
+            "clocks": clocks, "roofline": roofline, "kernels_alone": alone, "host_link": host_link,
+            "resume_latency_8k": lone,
+            "cpu_baseline": {"value": cpu["gbs"], "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample,
+                             "suspend_s": cpu["suspend_s"], "resume_s": cpu["resume_s"]},
+        }
+        print(json.dumps(out))
+    pool.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama3_8b", choices=list(CONFIGS))
+    ap.add_argument("--route", default="staged", choices=["staged", "mapped"])
+    ap.add_argument("--kernel", default="bulk", choices=["warp", "bulk"])
+    ap.add_argument("--chunk-mib", type=int, default=512)
+    ap.add_argument("--slots", type=int, default=2)
+    ap.add_argument("--max-ctas", type=int, default=0, help="cap on the movers' grid (0 = fill the GPU)")
+    ap.add_argument("--num-blocks", type=int, default=0, help="shrink the pool (profiling captures)")
+    ap.add_argument("--requests", type=int, default=0, help="override the request count")
+    ap.add_argument("--fixed-tokens", type=int, default=0, help="give every request this many tokens")
+    ap.add_argument("--no-extras", action="store_true", help="skip kernels-alone, lone-request and CPU legs")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -76,7 +76,7 @@ enum {
 #define KVR_SYNC 1u                  /* wait for the enqueued moves before returning */
 /* pool flags (kvr_config.flags) */
 #define KVR_METADATA_ONLY 1u         /* bookkeeping only: no buffers, no CUDA calls, nothing moves */
-#define KVR_PROFILE 2u               /* bracket every mover launch with timing events (kvr_stats.kernel_ms_*) */
+#define KVR_PROFILE 2u               /* bracket every mover launch with timing events (gather_ms, scatter_ms) */
 
 #define KVR_ROUTE_STAGED 1           /* kernel <-> HBM staging ring <-> chunked cudaMemcpyAsync */
 #define KVR_ROUTE_MAPPED 2           /* kernel reads / writes the pinned arena directly over the host link */
@@ -94,10 +94,10 @@ typedef struct {
   int32_t num_blocks;
   int32_t device;                    /* CUDA device ordinal */
   uint64_t host_capacity_bytes;      /* host tier budget */
-  uint64_t chunk_bytes;              /* staging slot size, multiple of 4096; 0 = 64 MiB */
-  int32_t staging_slots;             /* slots per direction; 0 = 3 */
+  uint64_t chunk_bytes;              /* staging slot size = largest chunk, multiple of 4096; 0 = 512 MiB */
+  int32_t staging_slots;             /* slots per direction, >= 2; 0 = 2 */
   int32_t route;                     /* KVR_ROUTE_*; 0 = KVR_ROUTE_STAGED */
-  int32_t kernel;                    /* KVR_KERNEL_*; 0 = KVR_KERNEL_WARP */
+  int32_t kernel;                    /* KVR_KERNEL_*; 0 = KVR_KERNEL_BULK */
   int32_t max_ctas;                  /* cap on the movers' grid (0 = fill the GPU) */
   uint32_t flags;                    /* KVR_METADATA_ONLY | KVR_PROFILE */
   uint32_t reserved;

@@ -76,6 +76,9 @@ __device__ __forceinline__ Tile locate(const MoveArgs &a, const long long *cum, 
 
 // ---- warp mover --------------------------------------------------------------------
 
+// One warp per tile; consecutive warps take consecutive tiles, so at any moment the grid covers one
+// contiguous window of the image.  A lane keeps 8 independent 16-byte loads in flight (streaming cache
+// policy: every byte is touched once) before it stores them.
 template <bool GATHER>
 __global__ void __launch_bounds__(kWarpThreads) move_warp_kernel(const MoveArgs a) {
   __shared__ long long cum[kMaxSegs + 1];
@@ -165,9 +168,12 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32) move_bulk_kernel(const Mov
   const int warps_per_cta = blockDim.x >> 5;
   const int pieces_per_tile = (a.tile_bytes + piece_bytes - 1) / piece_bytes;
   const long long total_units = a.total_tiles * pieces_per_tile;
+  // every pipeline takes one contiguous, equally long run of units
   const long long pipe = (long long)blockIdx.x * warps_per_cta + warp;
-  const long long stride = (long long)gridDim.x * warps_per_cta;
-  const long long n = pipe < total_units ? (total_units - pipe + stride - 1) / stride : 0;
+  const long long n_pipes = (long long)gridDim.x * warps_per_cta;
+  const long long per = total_units / n_pipes, extra = total_units - per * n_pipes;
+  const long long u0 = pipe * per + (pipe < extra ? pipe : extra);
+  const long long n = per + (pipe < extra ? 1 : 0);
   unsigned char *my_ring = ring + (size_t)warp * STAGES * piece_bytes;
   unsigned phase_bits = 0;
   bool failed = false;
@@ -177,7 +183,7 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32) move_bulk_kernel(const Mov
       const int stage = (int)(it % STAGES);
       // the store that last read this stage (unit it - STAGES) must be done with shared memory
       if (it >= STAGES) bulk_wait_read<STAGES - LAG - 1>();
-      const long long u = pipe + it * stride;
+      const long long u = u0 + it;
       const long long w = u / pieces_per_tile;
       const int off = (int)(u - w * pieces_per_tile) * piece_bytes;
       const Tile t = locate(a, cum, w);
@@ -244,9 +250,16 @@ cudaError_t opt_in(size_t smem) {
 cudaError_t launch_move_warp(bool gather, const MoveArgs &a, int grid_limit, int sm_count, cudaStream_t s) {
   if (a.total_tiles <= 0) return cudaSuccess;
   if (a.nsegs < 1 || a.nsegs > kMaxSegs) return cudaErrorInvalidValue;
+  static int ctas_per_sm = 0;                     // co-resident CTAs: the grid is one full wave, never more
+  if (!ctas_per_sm) {
+    int n = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, move_warp_kernel<true>, kWarpThreads, 0);
+    if (e != cudaSuccess) return e;
+    ctas_per_sm = n > 0 ? n : 1;
+  }
   const int warps_per_cta = kWarpThreads / 32;
   const long long work_ctas = (a.total_tiles + warps_per_cta - 1) / warps_per_cta;
-  const int grid = default_grid(grid_limit, sm_count, 2048 / kWarpThreads, work_ctas);
+  const int grid = default_grid(grid_limit, sm_count, ctas_per_sm, work_ctas);
   if (gather) move_warp_kernel<true><<<grid, kWarpThreads, 0, s>>>(a);
   else move_warp_kernel<false><<<grid, kWarpThreads, 0, s>>>(a);
   return cudaGetLastError();

@@ -20,6 +20,7 @@
 //   - a move on a request whose previous move is in flight waits for it.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <chrono>
 #include <cstdarg>
 #include <cstdio>
@@ -247,17 +248,38 @@ struct Plan {
   std::vector<int> req_chunk;     // item -> last chunk that holds bytes of it (-1: none)
 };
 
-// Staged route: cut the concatenated images into staging-slot sized chunks on tile boundaries.
-void plan_staged(kvr_pool *p, const std::vector<Item> &items, Ring &ring, const char *desc_dev, Plan &pl) {
-  const uint64_t cap = p->cfg.chunk_bytes;
+// Chunk sizes of one staged move.  A suspend starts with a small chunk and doubles up to the slot size,
+// so the first copy over the link starts after a few microseconds of gathering; a resume ends with
+// chunks that halve down to the small size, so little scattering is left after the last copy.  In
+// between, chunks are slot sized: few, large kernel launches.
+std::vector<uint64_t> chunk_caps(const kvr_pool *p, uint64_t total, bool ramp_up) {
+  const uint64_t big = p->cfg.chunk_bytes;
+  uint64_t small = 32ull << 20;
+  if (small < (uint64_t)p->tile_bytes) small = align_up(p->tile_bytes, 4096);
+  if (small > big) small = big;
+  std::vector<uint64_t> caps;
+  uint64_t sum = 0, c = small;
+  while (sum < total) { caps.push_back(c); sum += c; c = c * 2 > big ? big : c * 2; }
+  if (!ramp_up) std::reverse(caps.begin(), caps.end());
+  caps.push_back(small);      // chunks are cut on tile boundaries and may fall a little short: spare room
+  return caps;
+}
+
+// Staged route: cut the concatenated images into chunks on tile boundaries; chunk k goes to slot
+// (ring.next + k) mod slots and holds at most caps[k] bytes.
+void plan_staged(kvr_pool *p, const std::vector<Item> &items, Ring &ring, bool ramp_up, const char *desc_dev, Plan &pl) {
+  uint64_t total = 0;
+  for (auto &it : items) total += (uint64_t)it.n_tokens * p->bpt;
+  const std::vector<uint64_t> caps = chunk_caps(p, total, ramp_up);
   const int nslots = (int)ring.slots.size();
   Chunk cur;
-  uint64_t fill = 0;
+  uint64_t fill = 0, cap = caps[0];
   auto open = [&]() {
     cur = Chunk();
     cur.slot = (ring.next + (int)pl.chunks.size()) % nslots;
     cur.seg_begin = pl.segs.size();
     fill = 0;
+    cap = caps[pl.chunks.size() < caps.size() ? pl.chunks.size() : caps.size() - 1];
   };
   auto flush = [&]() {
     if (cur.nsegs) { cur.bytes = fill; pl.chunks.push_back(cur); }
@@ -367,7 +389,7 @@ kvr_status enqueue(kvr_pool *p, int kind, std::vector<Item> &items, int route, c
   Ring *ring = nullptr;
   if (route == KVR_ROUTE_STAGED) {
     ring = to_linear ? &p->out_ring : &p->in_ring;
-    plan_staged(p, items, *ring, nullptr, pl);
+    plan_staged(p, items, *ring, to_linear, nullptr, pl);
   } else {
     plan_direct(p, items, route == KVR_ROUTE_MAPPED ? p->arena_dev : lin_dev, nullptr, pl);
   }
@@ -549,8 +571,8 @@ kvr_status create_engine(kvr_pool *p) {
   CU(cudaHostAlloc((void **)&p->status_word, 64, cudaHostAllocMapped));
   *p->status_word = 0;
   if (c.kernel == KVR_KERNEL_BULK) {
-    int piece = p->tile_bytes < 16384 ? p->tile_bytes : 16384;
-    p->bulk = BulkShape{4, 3, piece};
+    int piece = p->tile_bytes < 32768 ? p->tile_bytes : 32768;
+    p->bulk = BulkShape{2, 3, piece};
     if (const char *env = getenv("KVR_BULK_SHAPE")) {   // "warps,stages,piece_bytes": tuning knob for benchmarks
       int w, s, b;
       if (sscanf(env, "%d,%d,%d", &w, &s, &b) == 3) p->bulk = BulkShape{w, s, b};
@@ -595,10 +617,10 @@ kvr_status kvr_pool_create(const kvr_config *cfg, kvr_pool **out) {
   kvr_pool *p = new (std::nothrow) kvr_pool();
   if (!p) return fail(KVR_ERR_NOMEM, "out of host memory");
   p->cfg = *cfg;
-  if (!p->cfg.chunk_bytes) p->cfg.chunk_bytes = 64ull << 20;
-  if (!p->cfg.staging_slots) p->cfg.staging_slots = 3;
+  if (!p->cfg.chunk_bytes) p->cfg.chunk_bytes = 512ull << 20;
+  if (!p->cfg.staging_slots) p->cfg.staging_slots = 2;
   if (!p->cfg.route) p->cfg.route = KVR_ROUTE_STAGED;
-  if (!p->cfg.kernel) p->cfg.kernel = KVR_KERNEL_WARP;
+  if (!p->cfg.kernel) p->cfg.kernel = KVR_KERNEL_BULK;
   kvr_status bad = KVR_OK;
   if (p->cfg.route != KVR_ROUTE_STAGED && p->cfg.route != KVR_ROUTE_MAPPED) bad = fail(KVR_ERR_INVALID_ARG, "unknown route");
   else if (p->cfg.kernel != KVR_KERNEL_WARP && p->cfg.kernel != KVR_KERNEL_BULK) bad = fail(KVR_ERR_INVALID_ARG, "unknown kernel");
