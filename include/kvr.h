@@ -215,6 +215,29 @@ kvr_status kvr_import_from_device(kvr_pool *pool, const uint64_t *req, int32_t n
                                   uint64_t capacity, uint64_t *offsets, uint32_t flags);
 
 /*
+ * The paper has no counterpart to this call; it exists for integration.  Some callers cannot allocate
+ * device memory: a serving engine that has given all of HBM to its own block allocator, or a
+ * latency-critical path that must not hit the device-wide synchronisation an allocation implies.
+ * This is kvr_export_to_device for ONE request without a pool handle and without any allocation: the
+ * segment record and the block table the gather kernel reads are copied into a fixed array in the
+ * library's device image (about 256 KiB, held by every GPU that loads the library until exit), so a
+ * request may have at most KVR_NOALLOC_MAX_BLOCKS blocks; more is rejected with KVR_ERR_INVALID_ARG
+ * and a message that names the limit.
+ *   device_pool : DEVICE, layout of the pool above, 16-byte aligned
+ *   block_table : HOST, nb = ceil(n_tokens / block_size) ids in [0, num_blocks)
+ *   dst_device  : DEVICE, n_tokens * kvr_bytes_per_token(g) bytes, 16-byte aligned
+ *   stream      : cudaStream_t (NULL = default stream); the work is enqueued, not waited for
+ * Runs on the current device.  The first call on each device looks up the array's address; make that
+ * call before starting any stream capture.  All calls share the array: calls whose GPU work may overlap
+ * (different streams or threads) race on it -- keep them on one stream or wait in between.  Nothing in
+ * the array needs clearing: each call overwrites what it uses.
+ */
+#define KVR_NOALLOC_MAX_BLOCKS 65536
+kvr_status kvr_gather_noalloc(const void *device_pool, const kvr_geometry *g, int32_t num_blocks,
+                              const int32_t *block_table, int32_t nb, int64_t n_tokens,
+                              void *dst_device, void *stream);
+
+/*
  * Observe one request.  Any out pointer may be NULL.  blocks (cap entries) is
  * written for requests that hold blocks; host_image is a borrowed pointer into
  * the arena, valid while the request stays in HOST; arena_offset is its offset.

@@ -36,6 +36,8 @@
 
 using namespace kvr;
 
+namespace kvr { void set_last_error(const char *msg); }
+
 namespace {
 
 thread_local std::string g_err;
@@ -49,6 +51,13 @@ kvr_status fail(kvr_status st, const char *fmt, ...) {
   g_err = buf;
   return st;
 }
+
+}  // namespace
+
+// lets the library's other source files report through kvr_last_error()
+void kvr::set_last_error(const char *msg) { g_err = msg ? msg : ""; }
+
+namespace {
 
 #define CU(call)                                                                              \
   do {                                                                                        \

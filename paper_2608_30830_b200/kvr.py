@@ -57,7 +57,7 @@ EXPORTS = [
     "kvr_retain_in_hbm", "kvr_suspend_to_host", "kvr_expire", "kvr_resume_from_host",
     "kvr_resume_from_host_into", "kvr_export_to_device", "kvr_import_from_device", "kvr_request_info",
     "kvr_request_latency", "kvr_wait", "kvr_pool_stats", "kvr_free_queue", "kvr_pool_device_ptr",
-    "kvr_pool_host_arena", "kvr_last_error",
+    "kvr_pool_host_arena", "kvr_last_error", "kvr_gather_noalloc",
 ]
 
 _lib = None
@@ -117,6 +117,8 @@ def lib():
     L.kvr_pool_host_arena.argtypes = [vp]
     L.kvr_last_error.restype = C.c_char_p
     L.kvr_last_error.argtypes = []
+    L.kvr_gather_noalloc.restype = i32
+    L.kvr_gather_noalloc.argtypes = [vp, C.POINTER(Geometry), i32, pi32, i32, i64, vp, vp]
     _lib = L
     return L
 
@@ -128,6 +130,18 @@ def last_error():
 def bytes_per_token(layers, kv_heads, head_dim, dtype_bytes, block_size=16):
     g = Geometry(layers, kv_heads, head_dim, dtype_bytes, block_size)
     return int(lib().kvr_bytes_per_token(C.byref(g)))
+
+
+NOALLOC_MAX_BLOCKS = 65536
+
+
+def gather_noalloc(device_pool, geom, num_blocks, block_table, n_tokens, dst_device, stream=None):
+    """kvr_gather_noalloc: one request's image, pool -> dst, with no allocation anywhere (see include/kvr.h).
+    geom = (layers, kv_heads, head_dim, dtype_bytes, block_size); block_table is a host int32 array."""
+    g = Geometry(*geom)
+    bt = np.ascontiguousarray(block_table, dtype=np.int32)
+    return lib().kvr_gather_noalloc(device_pool, C.byref(g), num_blocks, _i32p(bt) if bt.size else None, bt.size,
+                                    n_tokens, dst_device, stream)
 
 
 def _i32p(a):

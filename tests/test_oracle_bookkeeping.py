@@ -245,7 +245,7 @@ def test_suspend_does_not_touch_the_pool_and_image_is_logical_content():
 
 
 @settings(max_examples=60, deadline=None)
-@given(st.integers(0, 2**31), st.lists(st.integers(0, 40), min_size=1, max_size=5))
+@given(st.integers(0, 2**31), st.lists(st.integers(0, 36), min_size=1, max_size=5))
 def test_round_trip_under_any_relabelling(seed, lengths):
     NB = 48
     rng = np.random.default_rng(seed)
