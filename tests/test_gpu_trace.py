@@ -1,0 +1,126 @@
+"""The mixed tiering trace (retain / suspend / expire / resume events) on the GPU.
+
+Small geometry: the CPU oracle carries the data too, so every host image and the final pool are compared byte for
+byte.  Full geometry (Llama-3-8B-shaped KV, 256 requests, 48 GiB pool): the oracle carries the bookkeeping only and
+is compared call by call; the data is checked by content -- every admitted request's blocks are stamped with a
+pattern that encodes (request, plane, logical block, position), and the pattern must be intact, under the new
+block table, whenever a request comes back from the host."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from common import check_invariants
+from gpu_common import Twin
+from kvr_synth import CONFIGS, context_lengths, event_trace
+from paper_2608_30830_b200 import kvr
+from trace_driver import TraceRunner, host_ttl, mixture_mean
+
+pytestmark = [pytest.mark.gpu, pytest.mark.skipif(not torch.cuda.is_available(), reason="needs a CUDA device")]
+
+
+def thresholds(lengths, bpt, host_cap):
+    c2 = host_cap / (float(np.mean(lengths)) * bpt)
+    w_ref = mixture_mean()
+    lam = 2 * c2 / w_ref                          # the paper's 2 x lambda_crit operating point
+    return lam, host_ttl(lam, c2, w_ref)
+
+
+@pytest.mark.parametrize("mode", [dict(route=kvr.ROUTE_STAGED, kernel=kvr.KERNEL_BULK),
+                                  dict(route=kvr.ROUTE_MAPPED, kernel=kvr.KERNEL_WARP)], ids=["staged-bulk", "mapped-warp"])
+def test_trace_small_geometry_with_data(mode):
+    geom = (2, 2, 16, 2, 4)                        # 64-byte rows, 256 bytes per token
+    n_req, NB, host_cap = 160, 130, 160 * 4096
+    lengths = context_lengths(("lognormal", 64, 0.6, 4, 400), n_req, 21)
+    lam, ttl = thresholds(lengths, 256, host_cap)
+    events, _ = event_trace(n_req, 21, lam, 60.0, ttl)
+    t = Twin(geom, NB, host_cap, seed=21, chunk_bytes=8192, staging_slots=2, **mode)
+    rng = np.random.default_rng(21)
+    L, H, D, e, BS = geom
+    o_view = t.o.data.reshape(2 * L, NB, BS * H * D * e)
+    d_view = t.dev.view(2 * L, NB, BS * H * D * e)
+
+    def fill(rid, blocks, n):                      # new content for every admission, same bytes on both sides
+        if len(blocks) == 0:
+            return
+        fresh = rng.integers(0, 256, size=(2 * L, len(blocks), BS * H * D * e), dtype=np.uint8)
+        o_view[:, blocks] = fresh
+        d_view[:, torch.from_numpy(blocks.astype(np.int64)).cuda()] = torch.from_numpy(fresh).cuda()
+        torch.cuda.synchronize()
+
+    def after(name, args):
+        if name == "suspend_to_host":
+            t.assert_same_images(args[0])
+    counts = TraceRunner([t.o, t.g], lengths, fill=fill, after_call=after).run(events)
+    for k in ("offloaded", "resumed_resident", "resumed_from_host", "recomputed", "ttl_expired", "demoted"):
+        assert counts.get(k, 0) > 0, (k, counts)
+    t.assert_same_pool()
+    check_invariants(t.g, range(n_req))
+    t.close()
+
+
+def test_config4_trace_full_geometry():
+    w = CONFIGS["trace"]
+    seed = 20260830 + 3
+    L, H, D, e, BS = w.geom
+    bpt = kvr.bytes_per_token(L, H, D, e)
+    lengths = context_lengths(w.length_rule, w.n_requests, seed)
+    host_cap = 32 << 30
+    lam, ttl = thresholds(lengths, bpt, host_cap)
+    events, _ = event_trace(w.n_requests, seed, lam, 60.0, ttl)
+    NB = w.num_blocks
+    tile_words = BS * H * D * e // 8
+    dev = torch.zeros(NB * BS * bpt // 8, dtype=torch.int64, device="cuda")
+    view = dev.view(2 * L, NB, tile_words)
+    order = np.random.default_rng(seed).permutation(NB).astype(np.int32)
+    o = orc.OrcPool(*w.geom, NB, host_cap, initial_free_order=order, with_data=False)
+    g = kvr.Pool(*w.geom, NB, host_cap, initial_free_order=order, device_pool=dev.data_ptr())
+    plane_ix = torch.arange(2 * L, device="cuda", dtype=torch.int64).view(-1, 1, 1)
+    word_ix = torch.arange(tile_words, device="cuda", dtype=torch.int64).view(1, 1, -1)
+    epoch = {}
+
+    def pattern(rid, nb):
+        blk_ix = torch.arange(nb, device="cuda", dtype=torch.int64).view(1, -1, 1)
+        return ((rid + 1000 * epoch[rid]) << 40) ^ (plane_ix << 32) ^ (blk_ix << 12) ^ word_ix
+
+    def fill(rid, blocks, n):
+        epoch[rid] = epoch.get(rid, 0) + 1          # a recomputed request gets new content
+        if len(blocks):
+            view[:, torch.from_numpy(blocks.astype(np.int64)).cuda()] = pattern(rid, len(blocks))
+            torch.cuda.synchronize()                # the library's streams do not wait for torch's
+
+    checked = [0]
+
+    def verify(rid):
+        assert g.wait(rid) == kvr.OK, kvr.last_error()
+        d = g.info(rid)[1]
+        n, blocks = d["n_tokens"], d["blocks"]
+        if len(blocks) == 0:
+            return
+        got = view[:, torch.from_numpy(blocks.astype(np.int64)).cuda()]
+        want = pattern(rid, len(blocks))
+        full = n // BS                              # whole blocks: every word; last partial block: valid rows only
+        assert torch.equal(got[:, :full], want[:, :full]), "request %d came back changed" % rid
+        if full < len(blocks):
+            valid_words = (n - full * BS) * H * D * e // 8
+            assert torch.equal(got[:, full, :valid_words], want[:, full, :valid_words])
+        checked[0] += 1
+
+    steps = [0]
+
+    def after(name, args):
+        steps[0] += 1
+        if steps[0] % 16 == 0:                      # bookkeeping is compared on every call; the O(N) sweeps every 16th
+            check_invariants(g, range(w.n_requests))
+            assert o.free_queue().tolist() == g.free_queue().tolist()
+    counts = TraceRunner([o, g], lengths, fill=fill, verify=verify, after_call=after).run(events)
+    assert g.wait() == kvr.OK, kvr.last_error()
+    check_invariants(g, range(w.n_requests))
+    so, sg = o.stats(), g.stats()
+    for k in so:
+        assert so[k] == sg[k], k
+    assert counts["arrived"] == w.n_requests and counts.get("resumed_from_host", 0) > 50 and checked[0] > 100
+    assert sg["bytes_suspended"] - sg["bytes_resumed"] - sg["bytes_expired_from_host"] == 0 and sg["host_used"] == 0
+    print("config 4 trace:", counts, "GB suspended %.1f resumed %.1f" % (sg["bytes_suspended"] / 1e9, sg["bytes_resumed"] / 1e9))
+    g.close()
+    o.close()
