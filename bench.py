@@ -172,33 +172,148 @@ def link_peak(torch, kvr_pool, arena_bytes, reps=10):
     return out
 
 
-def run_ours(args):
+def run_longctx(args):
+    """Long-context stress: half of the 128k-token requests are suspended while the other half resumes, on the
+    library's two stream pairs, with and without a synthetic HBM-read load kernel running beside them."""
     import torch
-    import torch.distributed as dist
 
     from paper_2608_30830_b200 import kvr
+    from paper_2608_30830_b200.multi import env_ranks
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = env_ranks()
+    if rank != 0:
+        return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    w = CONFIGS["longctx"]
+    seed = SEED + 4
+    L, H, D, e, BS = w.geom
+    bpt = kvr.bytes_per_token(L, H, D, e)
+    n_tok = w.length_rule[1]
+    n_req = args.requests or w.n_requests
+    avail = int(open("/proc/meminfo").read().split("MemAvailable:")[1].split()[0]) * 1024
+    free_dev, _ = torch.cuda.mem_get_info()
+    load_bytes = 8 << 30
+    while n_req > 2 and (n_req * n_tok * bpt + (16 << 30) > 0.75 * avail or
+                         n_req * n_tok * bpt + load_bytes + (6 << 30) > free_dev):
+        n_req -= 2
+    NB = n_req * (n_tok // BS)
+    host_cap = n_req * n_tok * bpt + (64 << 20)
+    dev_pool = torch.empty(NB * BS * bpt, dtype=torch.uint8, device="cuda")
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    view = dev_pool.view(torch.bfloat16)
+    for i in range(0, view.numel(), 1 << 28):
+        view[i:i + (1 << 28)].normal_(generator=gen)
+    load_buf = torch.empty(load_bytes, dtype=torch.uint8, device="cuda").fill_(3)
+    sink = torch.zeros(1024, dtype=torch.int64, device="cuda")
+    torch.cuda.synchronize()
+    pool = kvr.Pool(*w.geom, NB, host_cap, initial_free_order=free_order(seed, NB), device=local,
+                    device_pool=dev_pool.data_ptr(), chunk_bytes=args.chunk_mib << 20, staging_slots=args.slots,
+                    kernel={"warp": kvr.KERNEL_WARP, "bulk": kvr.KERNEL_BULK}[args.kernel], max_ctas=args.max_ctas,
+                    flags=kvr.PROFILE)
+    ids = list(range(n_req))
+    for rid in ids:
+        assert pool.admit(rid, n_tok)[0] == kvr.OK
+    on_host, in_hbm = ids[:n_req // 2], ids[n_req // 2:]
+    assert pool.suspend_to_host(on_host, kvr.SYNC)[0] == kvr.OK            # phase A, untimed
+    half_bytes = (n_req // 2) * n_tok * bpt
+    load_stream = torch.cuda.Stream()
 
-    # scale rule: every rank pins its own arena out of the same host DRAM; keep geometry and lengths,
-    # reduce the request count when the arenas of all ranks would not fit in 60% of what is available
+    def load_rate(launches):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(load_stream):
+            e0.record()
+            assert kvr.read_load(load_buf.data_ptr(), load_bytes, launches, sink.data_ptr(), load_stream.cuda_stream) == kvr.OK
+            e1.record()
+        return e0, e1, launches * load_bytes
+
+    def exchange(overlap, load_launches):
+        nonlocal on_host, in_hbm
+        ev = load_rate(load_launches) if load_launches else None
+        t0 = time.perf_counter()
+        assert pool.suspend_to_host(in_hbm)[0] == kvr.OK
+        if not overlap:
+            assert pool.wait() == kvr.OK
+        assert pool.resume_from_host(on_host)[0] == kvr.OK
+        assert pool.wait() == kvr.OK, kvr.last_error()
+        wall = time.perf_counter() - t0
+        sus = max(pool.latency(r)[2] for r in in_hbm) / 1e3
+        res = max(pool.latency(r)[2] for r in on_host) / 1e3
+        out = {"suspend_gbs": half_bytes / sus / 1e9, "resume_gbs": half_bytes / res / 1e9,
+               "both_directions_gbs": 2 * half_bytes / wall / 1e9, "wall_s": wall}
+        if ev:
+            torch.cuda.synchronize()
+            out["load_gbs"] = ev[2] / ev[0].elapsed_time(ev[1]) / 1e6
+        on_host, in_hbm = in_hbm, on_host
+        return out
+
+    def median_of(runs):
+        return {k: float(np.median([r[k] for r in runs])) for k in runs[0]}
+
+    exchange(True, 0)                                                      # warm-up
+    e0, e1, nb = load_rate(200)
+    torch.cuda.synchronize()
+    load_alone = nb / e0.elapsed_time(e1) / 1e6
+    sampler = ClockSampler(local)
+    sampler.start()
+    reps = max(args.steps, 1)
+    seq = median_of([exchange(False, 0) for _ in range(reps)])
+    ovl = median_of([exchange(True, 0) for _ in range(reps)])
+    # size the load so that it runs for most of the overlapped exchange
+    launches = max(50, int(0.8 * ovl["wall_s"] * load_alone * 1e9 / load_bytes))
+    ovl_load = median_of([exchange(True, launches) for _ in range(reps)])
+    clocks = sampler.stop()
+    st = pool.stats()
+    peak, peak_kind = peaks()
+    link = link_peak(torch, pool, host_cap)
+    out = {
+        "metric": "suspend/resume payload GB/s, both directions overlapped beside a synthetic HBM-read load",
+        "value": ovl_load["both_directions_gbs"], "unit": "GB/s", "n_gpus": 1, "steps": reps, "warmup": 1,
+        "ms_per_step": 1e3 * ovl_load["wall_s"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u8", "data": "synthetic",
+        "config": {"workload": "longctx", "geometry": dict(zip(("layers", "kv_heads", "head_dim", "dtype_bytes", "block_size"), w.geom)),
+                   "requests_requested": w.n_requests, "requests_run": n_req, "tokens_per_request": n_tok,
+                   "bytes_per_direction": half_bytes, "num_blocks": NB, "load_buffer_bytes": load_bytes,
+                   "kernel": args.kernel, "chunk_mib": args.chunk_mib, "max_ctas": args.max_ctas},
+        "interference": {
+            "alone_one_direction_at_a_time": seq, "overlapped": ovl, "overlapped_with_load": ovl_load,
+            "load_alone_gbs": load_alone, "load_alone_frac_of_hbm_peak": load_alone / peak,
+            "suspend_loss_pct_overlap": 100 * (1 - ovl["suspend_gbs"] / seq["suspend_gbs"]),
+            "resume_loss_pct_overlap": 100 * (1 - ovl["resume_gbs"] / seq["resume_gbs"]),
+            "suspend_loss_pct_overlap_and_load": 100 * (1 - ovl_load["suspend_gbs"] / seq["suspend_gbs"]),
+            "resume_loss_pct_overlap_and_load": 100 * (1 - ovl_load["resume_gbs"] / seq["resume_gbs"]),
+            "load_loss_pct": 100 * (1 - ovl_load["load_gbs"] / load_alone)},
+        "host_link": link, "clocks": clocks,
+        "gpu_launches": int(st["gather_launches"] + st["scatter_launches"]),
+    }
+    print(json.dumps(out))
+    pool.close()
+
+
+def run_ours(args):
+    import torch
+
+    from paper_2608_30830_b200 import kvr
+    from paper_2608_30830_b200.multi import Group, env_ranks, fit_requests
+
+    rank, world, local = env_ranks()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    group = Group("nccl", torch.device("cuda", local))
+
+    # every rank runs its own replica of the workload (own pool, own host link, own arena): weak scaling.
+    # Scale rule: the arenas of all ranks come out of the same host DRAM; keep geometry and lengths and
+    # reduce the request count when they would not fit in 60% of what is available.
     ov = {"num_blocks": args.num_blocks, "requests": args.requests, "fixed_tokens": args.fixed_tokens}
     w, seed, lens, fillers = build_workload(args.workload, None, ov)
     bpt = kvr.bytes_per_token(*w.geom[:4])
     requested = len(lens)
     avail = int(open("/proc/meminfo").read().split("MemAvailable:")[1].split()[0]) * 1024
-    budget = int(0.6 * avail / world)
-    while len(lens) > 1 and int(lens.sum()) * bpt + (2 << 30) > budget:
-        lens = lens[:-1]
-    if len(lens) != requested:
-        w, seed, lens, fillers = build_workload(args.workload, len(lens), ov)
+    keep = int(group.max([-fit_requests(lens, bpt, avail, world)])[0]) * -1      # the same count on every rank
+    if keep != requested:
+        w, seed, lens, fillers = build_workload(args.workload, keep, ov)
     L, H, D, e, BS = w.geom
     payload = int(lens.sum()) * bpt
     lone_tokens = 8192
@@ -239,8 +354,7 @@ def run_ours(args):
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        group.barrier()
 
     def one_step():
         """Returns (device_ms_suspend, device_ms_resume, wall_s)."""
@@ -279,15 +393,8 @@ def run_ours(args):
     sus_ms = float(np.sum([s[0] for s in steps]))
     res_ms = float(np.sum([s[1] for s in steps]))
     dev_s = (sus_ms + res_ms) / 1e3
-    if world > 1:
-        tt = torch.tensor([dev_s, wall, sus_ms, res_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        dev_s, wall, sus_ms, res_ms = tt.tolist()
-        pp = torch.tensor([payload], dtype=torch.float64, device="cuda")
-        dist.all_reduce(pp, op=dist.ReduceOp.SUM)
-        payload_all = float(pp.item())
-    else:
-        payload_all = float(payload)
+    dev_s, wall, sus_ms, res_ms = group.max([dev_s, wall, sus_ms, res_ms])    # the job is as slow as its slowest rank
+    payload_all = group.sum([payload])[0]
     K = args.steps
     moved = 2.0 * payload_all * K                      # bytes suspended + bytes resumed, all ranks
     value = moved / dev_s / 1e9
@@ -386,9 +493,7 @@ def run_ours(args):
         }
         print(json.dumps(out))
     pool.close()
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    group.close()
 
 
 def main():
@@ -410,6 +515,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "longctx":
+        run_longctx(args)
     else:
         run_ours(args)
 

@@ -260,6 +260,14 @@ kvr_status kvr_request_latency(kvr_pool *pool, uint64_t req, double *host_ms, do
  */
 kvr_status kvr_wait(kvr_pool *pool, uint64_t req_or_all, int64_t timeout_ms);
 
+/*
+ * Benchmark support, not part of the method: the synthetic competing load of the long-context interference
+ * measurement.  Enqueues `launches` kernels on `stream` (a cudaStream_t), each streaming the DEVICE buffer
+ * (bytes, 16-byte aligned) once out of HBM in short-lived CTAs; device_sink is 8 KiB of DEVICE memory the
+ * kernels fold what they read into.  Returns at once; time it with events on `stream`.
+ */
+kvr_status kvr_read_load(const void *device_buf, uint64_t bytes, int32_t launches, void *device_sink, void *stream);
+
 kvr_status kvr_pool_stats(kvr_pool *pool, kvr_stats *out);
 /* copies the free queue, head first, into out (cap entries, may be NULL); returns its length */
 int64_t kvr_free_queue(kvr_pool *pool, int32_t *out, int64_t cap);

@@ -220,6 +220,24 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32) move_bulk_kernel(const Mov
   bulk_wait_all();
 }
 
+// Synthetic competing load: every CTA streams one 32 KiB slice of a large buffer and folds it into a sink word.
+// CTAs are short-lived on purpose, so higher-priority mover CTAs get SM slots as these retire.
+__global__ void __launch_bounds__(256) read_load_kernel(const uint4 *buf, unsigned long long nvec, unsigned long long *sink) {
+  const unsigned long long base = (unsigned long long)blockIdx.x * (256 * 8) + threadIdx.x;
+  uint4 v[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const unsigned long long i = base + 256ull * k;
+    v[k] = i < nvec ? __ldcs(buf + i) : make_uint4(0, 0, 0, 0);
+  }
+  unsigned acc = 0;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) acc ^= v[k].x ^ v[k].y ^ v[k].z ^ v[k].w;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) acc ^= __shfl_xor_sync(0xffffffffu, acc, d);
+  if ((threadIdx.x & 31) == 0) atomicXor(sink + (blockIdx.x & 1023), (unsigned long long)acc);
+}
+
 int default_grid(int grid_limit, int sm_count, int ctas_per_sm, long long work_ctas) {
   long long g = (long long)sm_count * ctas_per_sm;
   if (grid_limit > 0 && g > grid_limit) g = grid_limit;
@@ -262,6 +280,15 @@ cudaError_t launch_move_warp(bool gather, const MoveArgs &a, int grid_limit, int
   const int grid = default_grid(grid_limit, sm_count, ctas_per_sm, work_ctas);
   if (gather) move_warp_kernel<true><<<grid, kWarpThreads, 0, s>>>(a);
   else move_warp_kernel<false><<<grid, kWarpThreads, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_read_load(const void *buf, unsigned long long bytes, int launches, void *sink, cudaStream_t s) {
+  const unsigned long long nvec = bytes >> 4;
+  const unsigned long long ctas = (nvec + 256 * 8 - 1) / (256 * 8);
+  if (ctas < 1 || ctas > 0x7fffffffull) return cudaErrorInvalidValue;
+  for (int i = 0; i < launches; ++i)
+    read_load_kernel<<<(unsigned)ctas, 256, 0, s>>>(static_cast<const uint4 *>(buf), nvec, static_cast<unsigned long long *>(sink));
   return cudaGetLastError();
 }
 

@@ -46,4 +46,7 @@ cudaError_t launch_move_bulk(bool gather, const MoveArgs &a, const BulkShape &sh
                              int sm_count, cudaStream_t s);
 cudaError_t bulk_configure(const BulkShape &shape);   // once per device: opt in to large dynamic shared memory
 
+// `launches` back-to-back streaming reads of buf (benchmark load); sink = 8 KiB of device memory
+cudaError_t launch_read_load(const void *buf, unsigned long long bytes, int launches, void *sink, cudaStream_t s);
+
 }  // namespace kvr

@@ -943,6 +943,14 @@ int64_t kvr_free_queue(kvr_pool *p, int32_t *out, int64_t cap) {
   return n;
 }
 
+kvr_status kvr_read_load(const void *device_buf, uint64_t bytes, int32_t launches, void *device_sink, void *stream) {
+  if (!device_buf || !device_sink || bytes < 16 || launches < 0 || ((uintptr_t)device_buf & 15) || ((uintptr_t)device_sink & 7))
+    return fail(KVR_ERR_INVALID_ARG, "kvr_read_load: NULL, misaligned or empty buffer");
+  cudaError_t e = launch_read_load(device_buf, bytes, launches, device_sink, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fail(KVR_ERR_CUDA, "read load launch: %s", cudaGetErrorString(e));
+  return KVR_OK;
+}
+
 void *kvr_pool_device_ptr(kvr_pool *p) { return p ? p->d_pool : nullptr; }
 void *kvr_pool_host_arena(kvr_pool *p) { return p ? p->h_arena : nullptr; }
 

@@ -57,7 +57,7 @@ EXPORTS = [
     "kvr_retain_in_hbm", "kvr_suspend_to_host", "kvr_expire", "kvr_resume_from_host",
     "kvr_resume_from_host_into", "kvr_export_to_device", "kvr_import_from_device", "kvr_request_info",
     "kvr_request_latency", "kvr_wait", "kvr_pool_stats", "kvr_free_queue", "kvr_pool_device_ptr",
-    "kvr_pool_host_arena", "kvr_last_error", "kvr_gather_noalloc",
+    "kvr_pool_host_arena", "kvr_last_error", "kvr_gather_noalloc", "kvr_read_load",
 ]
 
 _lib = None
@@ -117,6 +117,8 @@ def lib():
     L.kvr_pool_host_arena.argtypes = [vp]
     L.kvr_last_error.restype = C.c_char_p
     L.kvr_last_error.argtypes = []
+    L.kvr_read_load.restype = i32
+    L.kvr_read_load.argtypes = [vp, u64, i32, vp, vp]
     L.kvr_gather_noalloc.restype = i32
     L.kvr_gather_noalloc.argtypes = [vp, C.POINTER(Geometry), i32, pi32, i32, i64, vp, vp]
     _lib = L
@@ -130,6 +132,11 @@ def last_error():
 def bytes_per_token(layers, kv_heads, head_dim, dtype_bytes, block_size=16):
     g = Geometry(layers, kv_heads, head_dim, dtype_bytes, block_size)
     return int(lib().kvr_bytes_per_token(C.byref(g)))
+
+
+def read_load(device_buf, nbytes, launches, device_sink, stream=None):
+    """kvr_read_load: enqueue the synthetic HBM-read load (benchmark support)."""
+    return lib().kvr_read_load(device_buf, nbytes, launches, device_sink, stream)
 
 
 NOALLOC_MAX_BLOCKS = 65536

@@ -180,6 +180,24 @@ def test_transient_states_and_latency():
     t.close()
 
 
+def test_wait_is_bounded():
+    """kvr_wait with a zero budget on a move that is still in flight answers KVR_ERR_TIMEOUT at once and leaves
+    the move alone; a later wait sees it finish."""
+    geom = (32, 8, 128, 2, 16)
+    n = 4096                                                 # 512 MiB image: ~9 ms on the link
+    bpt = kvr.bytes_per_token(*geom[:4])
+    dev = torch.zeros(512 * 16 * bpt, dtype=torch.uint8, device="cuda")
+    with kvr.Pool(*geom, 512, n * bpt + 4096, device_pool=dev.data_ptr()) as g:
+        assert g.admit(1, n)[0] == kvr.OK
+        assert g.suspend_to_host([1])[0] == kvr.OK
+        st = g.wait(1, 0)
+        assert st in (kvr.ERR_TIMEOUT, kvr.OK)
+        if st == kvr.ERR_TIMEOUT:
+            assert "in flight" in kvr.last_error() and g.info(1)[1]["state"] == kvr.SUSPENDING
+        assert g.wait(1, 10000) == kvr.OK and g.info(1)[1]["state"] == kvr.HOST
+        assert g.stats()["ops_in_flight"] == 0
+
+
 def test_caller_owned_pinned_arena_and_grid_cap():
     geom = (4, 2, 64, 2, 16)
     cap = 1 << 21
