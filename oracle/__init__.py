@@ -7,5 +7,5 @@ from .orc import (  # noqa: F401
     OrcPool, OrcStats, build, bytes_per_token, gather, image_offset, pool_offset, scatter,
     OK, RESIDENT, RECOMPUTE, HOST_FULL, HBM_FULL,
     ERR_INVALID_ARG, ERR_UNKNOWN_REQUEST, ERR_BAD_STATE, ERR_GEOMETRY, ERR_NOMEM,
-    ACTIVE, RETAINED, HOST, EXPIRED,
+    ACTIVE, RETAINED, HOST, EXPIRED, LAYER_MAJOR, BLOCK_MAJOR,
 )

@@ -28,7 +28,7 @@ typedef struct {
 typedef struct { uint64_t off, len; uint64_t id; } orc_range;
 
 struct orc_pool {
-  int32_t L, H, D, e, BS, NB;
+  int32_t L, H, D, e, BS, NB, layout;
   uint64_t bpt;
   int32_t with_data;
   uint8_t *data;
@@ -52,12 +52,20 @@ uint64_t orc_bytes_per_token(int32_t layers, int32_t kv_heads, int32_t head_dim,
 }
 
 uint64_t orc_pool_offset(int32_t L, int32_t H, int32_t D, int32_t e, int32_t BS, int32_t NB,
-                         int32_t l, int32_t kv, int32_t blk, int32_t slot, int32_t h, int32_t d, int32_t byte) {
-  (void)L;
-  /* pool[L][2][NB][BS][H][D][e]: Horner form of the row-major index */
-  uint64_t i = (uint64_t)l;
-  i = i * 2u + (uint64_t)kv;
-  i = i * (uint64_t)NB + (uint64_t)blk;
+                         int32_t l, int32_t kv, int32_t blk, int32_t slot, int32_t h, int32_t d, int32_t byte,
+                         int32_t layout) {
+  uint64_t i;
+  if (layout == ORC_BLOCK_MAJOR) {
+    /* pool[NB][L][2][BS][H][D][e]: Horner form of the row-major index */
+    i = (uint64_t)blk;
+    i = i * (uint64_t)L + (uint64_t)l;
+    i = i * 2u + (uint64_t)kv;
+  } else {
+    /* pool[L][2][NB][BS][H][D][e] */
+    i = (uint64_t)l;
+    i = i * 2u + (uint64_t)kv;
+    i = i * (uint64_t)NB + (uint64_t)blk;
+  }
   i = i * (uint64_t)BS + (uint64_t)slot;
   i = i * (uint64_t)H + (uint64_t)h;
   i = i * (uint64_t)D + (uint64_t)d;
@@ -79,7 +87,7 @@ uint64_t orc_image_offset(int32_t L, int32_t H, int32_t D, int32_t e, int64_t n,
 }
 
 void orc_gather(const uint8_t *pool, uint8_t *image, int32_t L, int32_t H, int32_t D, int32_t e,
-                int32_t BS, int32_t NB, const int32_t *bt, int64_t n) {
+                int32_t BS, int32_t NB, const int32_t *bt, int64_t n, int32_t layout) {
   for (int32_t l = 0; l < L; ++l)
     for (int32_t kv = 0; kv < 2; ++kv)
       for (int64_t t = 0; t < n; ++t) {
@@ -89,12 +97,12 @@ void orc_gather(const uint8_t *pool, uint8_t *image, int32_t L, int32_t H, int32
           for (int32_t d = 0; d < D; ++d)
             for (int32_t b = 0; b < e; ++b)
               image[orc_image_offset(L, H, D, e, n, l, kv, t, h, d, b)] =
-                  pool[orc_pool_offset(L, H, D, e, BS, NB, l, kv, blk, slot, h, d, b)];
+                  pool[orc_pool_offset(L, H, D, e, BS, NB, l, kv, blk, slot, h, d, b, layout)];
       }
 }
 
 void orc_scatter(uint8_t *pool, const uint8_t *image, int32_t L, int32_t H, int32_t D, int32_t e,
-                 int32_t BS, int32_t NB, const int32_t *bt, int64_t n) {
+                 int32_t BS, int32_t NB, const int32_t *bt, int64_t n, int32_t layout) {
   for (int32_t l = 0; l < L; ++l)
     for (int32_t kv = 0; kv < 2; ++kv)
       for (int64_t t = 0; t < n; ++t) {
@@ -103,7 +111,7 @@ void orc_scatter(uint8_t *pool, const uint8_t *image, int32_t L, int32_t H, int3
         for (int32_t h = 0; h < H; ++h)
           for (int32_t d = 0; d < D; ++d)
             for (int32_t b = 0; b < e; ++b)
-              pool[orc_pool_offset(L, H, D, e, BS, NB, l, kv, blk, slot, h, d, b)] =
+              pool[orc_pool_offset(L, H, D, e, BS, NB, l, kv, blk, slot, h, d, b, layout)] =
                   image[orc_image_offset(L, H, D, e, n, l, kv, t, h, d, b)];
       }
 }
@@ -111,11 +119,13 @@ void orc_scatter(uint8_t *pool, const uint8_t *image, int32_t L, int32_t H, int3
 /* ---- pool --------------------------------------------------------------- */
 
 orc_pool *orc_pool_create(int32_t L, int32_t H, int32_t D, int32_t e, int32_t BS, int32_t NB,
-                          uint64_t host_capacity, const int32_t *initial_free_order, int32_t with_data) {
+                          uint64_t host_capacity, const int32_t *initial_free_order, int32_t with_data,
+                          int32_t layout) {
   if (orc_bytes_per_token(L, H, D, e) == 0 || BS < 1 || NB < 1) return NULL;
+  if (layout != ORC_LAYER_MAJOR && layout != ORC_BLOCK_MAJOR) return NULL;
   orc_pool *p = (orc_pool *)calloc(1, sizeof(orc_pool));
   if (!p) return NULL;
-  p->L = L; p->H = H; p->D = D; p->e = e; p->BS = BS; p->NB = NB;
+  p->L = L; p->H = H; p->D = D; p->e = e; p->BS = BS; p->NB = NB; p->layout = layout;
   p->bpt = orc_bytes_per_token(L, H, D, e);
   p->with_data = with_data;
   p->host_capacity = host_capacity;
@@ -295,7 +305,7 @@ static int32_t suspend_one(orc_pool *p, uint64_t id) {
   if (p->with_data) {
     r->image = (uint8_t *)malloc((size_t)(r->image_bytes ? r->image_bytes : 1));
     if (!r->image) { if (len) arena_remove(p, id); return ORC_ERR_NOMEM; }
-    orc_gather(p->data, r->image, p->L, p->H, p->D, p->e, p->BS, p->NB, r->blocks, r->n_tokens);
+    orc_gather(p->data, r->image, p->L, p->H, p->D, p->e, p->BS, p->NB, r->blocks, r->n_tokens, p->layout);
   }
   r->arena_off = off; r->arena_len = len;
   drop_blocks(p, r);                 /* ids go to the free tail in logical order */
@@ -322,7 +332,7 @@ static int32_t expire_one(orc_pool *p, uint64_t id) {
 
 static int32_t resume_with_blocks(orc_pool *p, orc_req *r, int32_t *blocks) {
   if (p->with_data)
-    orc_scatter(p->data, r->image, p->L, p->H, p->D, p->e, p->BS, p->NB, blocks, r->n_tokens);
+    orc_scatter(p->data, r->image, p->L, p->H, p->D, p->e, p->BS, p->NB, blocks, r->n_tokens, p->layout);
   drop_host_copy(p, r);
   r->blocks = blocks;
   r->state = ORC_ACTIVE;

@@ -58,6 +58,11 @@ typedef struct {
   uint64_t bytes_suspended, bytes_resumed, bytes_expired_from_host;
 } orc_stats;
 
+/* Pool layouts (the paper names none; both keep one (layer, plane, block) tile contiguous):
+ *   ORC_LAYER_MAJOR : bytes [L][2][NB][BS][H][D][e]   (the default reading)
+ *   ORC_BLOCK_MAJOR : bytes [NB][L][2][BS][H][D][e]   (all planes of a block adjacent) */
+enum { ORC_LAYER_MAJOR = 0, ORC_BLOCK_MAJOR = 1 };
+
 /* Appendix B closed form; 0 when any factor is < 1. */
 uint64_t orc_bytes_per_token(int32_t layers, int32_t kv_heads, int32_t head_dim, int32_t dtype_bytes);
 
@@ -65,14 +70,16 @@ uint64_t orc_bytes_per_token(int32_t layers, int32_t kv_heads, int32_t head_dim,
  * `blk` of plane kv of layer l in the pool array; and of token t in an image
  * of n tokens.  Written from the array declarations above, nothing else. */
 uint64_t orc_pool_offset(int32_t L, int32_t H, int32_t D, int32_t e, int32_t BS, int32_t NB,
-                         int32_t l, int32_t kv, int32_t blk, int32_t slot, int32_t h, int32_t d, int32_t byte);
+                         int32_t l, int32_t kv, int32_t blk, int32_t slot, int32_t h, int32_t d, int32_t byte,
+                         int32_t layout);
 uint64_t orc_image_offset(int32_t L, int32_t H, int32_t D, int32_t e, int64_t n,
                           int32_t l, int32_t kv, int64_t t, int32_t h, int32_t d, int32_t byte);
 
 /* with_data = 0: bookkeeping only (no pool bytes, no images).
  * initial_free_order: permutation of [0, NB) or NULL for identity. */
 orc_pool *orc_pool_create(int32_t L, int32_t H, int32_t D, int32_t e, int32_t BS, int32_t NB,
-                          uint64_t host_capacity, const int32_t *initial_free_order, int32_t with_data);
+                          uint64_t host_capacity, const int32_t *initial_free_order, int32_t with_data,
+                          int32_t layout);
 void orc_pool_destroy(orc_pool *);
 uint8_t *orc_pool_data(orc_pool *);      /* NULL when with_data = 0 */
 uint64_t orc_pool_bytes(orc_pool *);
@@ -97,9 +104,9 @@ int64_t orc_free_queue(orc_pool *, int32_t *out, int64_t cap);
 /* The two data movements on their own, for timing and for element checks:
  * image[l][kv][t][h][d] = pool[l][kv][bt[t / BS]][t % BS][h][d], and back. */
 void orc_gather(const uint8_t *pool, uint8_t *image, int32_t L, int32_t H, int32_t D, int32_t e,
-                int32_t BS, int32_t NB, const int32_t *bt, int64_t n);
+                int32_t BS, int32_t NB, const int32_t *bt, int64_t n, int32_t layout);
 void orc_scatter(uint8_t *pool, const uint8_t *image, int32_t L, int32_t H, int32_t D, int32_t e,
-                 int32_t BS, int32_t NB, const int32_t *bt, int64_t n);
+                 int32_t BS, int32_t NB, const int32_t *bt, int64_t n, int32_t layout);
 
 #ifdef __cplusplus
 }

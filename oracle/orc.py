@@ -16,6 +16,7 @@ _SRC = [os.path.join(_DIR, "kvr_oracle.c"), os.path.join(_DIR, "kvr_oracle.h")]
 OK, RESIDENT, RECOMPUTE, HOST_FULL, HBM_FULL = 0, 1, 2, 3, 4
 ERR_INVALID_ARG, ERR_UNKNOWN_REQUEST, ERR_BAD_STATE, ERR_GEOMETRY, ERR_NOMEM = -1, -2, -3, -4, -7
 ACTIVE, RETAINED, HOST, EXPIRED = 0, 1, 3, 5
+LAYER_MAJOR, BLOCK_MAJOR = 0, 1
 
 
 def build(force=False):
@@ -54,11 +55,11 @@ def lib():
         L.orc_bytes_per_token.restype = u64
         L.orc_bytes_per_token.argtypes = [i32] * 4
         L.orc_pool_offset.restype = u64
-        L.orc_pool_offset.argtypes = [i32] * 13
+        L.orc_pool_offset.argtypes = [i32] * 14
         L.orc_image_offset.restype = u64
         L.orc_image_offset.argtypes = [i32, i32, i32, i32, i64, i32, i32, i64, i32, i32, i32]
         L.orc_pool_create.restype = vp
-        L.orc_pool_create.argtypes = [i32] * 6 + [u64, pi32, i32]
+        L.orc_pool_create.argtypes = [i32] * 6 + [u64, pi32, i32, i32]
         L.orc_pool_destroy.restype = None
         L.orc_pool_destroy.argtypes = [vp]
         L.orc_pool_data.restype = vp
@@ -85,7 +86,7 @@ def lib():
         for name in ("orc_gather", "orc_scatter"):
             f = getattr(L, name)
             f.restype = None
-            f.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, pi32, i64]
+            f.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, pi32, i64, i32]
     return _lib
 
 
@@ -93,8 +94,8 @@ def bytes_per_token(layers, kv_heads, head_dim, dtype_bytes):
     return int(lib().orc_bytes_per_token(layers, kv_heads, head_dim, dtype_bytes))
 
 
-def pool_offset(L, H, D, e, BS, NB, l, kv, blk, slot, h=0, d=0, byte=0):
-    return int(lib().orc_pool_offset(L, H, D, e, BS, NB, l, kv, blk, slot, h, d, byte))
+def pool_offset(L, H, D, e, BS, NB, l, kv, blk, slot, h=0, d=0, byte=0, layout=LAYER_MAJOR):
+    return int(lib().orc_pool_offset(L, H, D, e, BS, NB, l, kv, blk, slot, h, d, byte, layout))
 
 
 def image_offset(L, H, D, e, n, l, kv, t, h=0, d=0, byte=0):
@@ -105,31 +106,33 @@ def _i32p(a):
     return a.ctypes.data_as(C.POINTER(C.c_int32))
 
 
-def gather(pool, L, H, D, e, BS, NB, bt, n):
+def gather(pool, L, H, D, e, BS, NB, bt, n, layout=LAYER_MAJOR):
     """image = gather(pool) for one request; pool is a flat uint8 array."""
     bt = np.ascontiguousarray(bt, dtype=np.int32)
     image = np.zeros(n * 2 * L * H * D * e, dtype=np.uint8)
-    lib().orc_gather(pool.ctypes.data, image.ctypes.data, L, H, D, e, BS, NB, _i32p(bt), n)
+    lib().orc_gather(pool.ctypes.data, image.ctypes.data, L, H, D, e, BS, NB, _i32p(bt), n, layout)
     return image
 
 
-def scatter(pool, image, L, H, D, e, BS, NB, bt, n):
+def scatter(pool, image, L, H, D, e, BS, NB, bt, n, layout=LAYER_MAJOR):
     bt = np.ascontiguousarray(bt, dtype=np.int32)
     image = np.ascontiguousarray(image, dtype=np.uint8)
-    lib().orc_scatter(pool.ctypes.data, image.ctypes.data, L, H, D, e, BS, NB, _i32p(bt), n)
+    lib().orc_scatter(pool.ctypes.data, image.ctypes.data, L, H, D, e, BS, NB, _i32p(bt), n, layout)
 
 
 class OrcPool:
     """One oracle pool.  Methods mirror the C-ABI call set of the product library."""
 
-    def __init__(self, L, H, D, e, BS, NB, host_capacity, initial_free_order=None, with_data=True):
+    def __init__(self, L, H, D, e, BS, NB, host_capacity, initial_free_order=None, with_data=True,
+                 layout=LAYER_MAJOR):
         self.geom = (L, H, D, e, BS)
         self.NB = NB
+        self.layout = layout
         order = None
         if initial_free_order is not None:
             order = np.ascontiguousarray(initial_free_order, dtype=np.int32)
         self._h = lib().orc_pool_create(L, H, D, e, BS, NB, host_capacity,
-                                        _i32p(order) if order is not None else None, int(with_data))
+                                        _i32p(order) if order is not None else None, int(with_data), layout)
         if not self._h:
             raise ValueError("orc_pool_create failed (geometry, free order or memory)")
         self.with_data = with_data

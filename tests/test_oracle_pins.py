@@ -163,3 +163,67 @@ def test_transposed_or_swapped_planes_would_fail():
             pool[l, kv] = 10 * l + kv + 1
     img = orc.gather(pool.reshape(-1), L, H, D, e, BS, NB, [2, 0], 3).reshape(L, 2, 3 * H * D * e)
     assert (img[0, 0] == 1).all() and (img[0, 1] == 2).all() and (img[1, 0] == 11).all() and (img[1, 1] == 12).all()
+
+
+# ---- block-major pool layout [NB][L][2][BS][H][D][e]: same pins ------------------------
+
+def test_block_major_offsets_match_numpy_strides():
+    rng = np.random.default_rng(3)
+    for _ in range(200):
+        L, H, D, e, BS, NB = (int(rng.integers(1, 5)) for _ in range(6))
+        l, kv = int(rng.integers(L)), int(rng.integers(2))
+        blk, slot, h, d, b = (int(rng.integers(x)) for x in (NB, BS, H, D, e))
+        assert orc.pool_offset(L, H, D, e, BS, NB, l, kv, blk, slot, h, d, b, layout=orc.BLOCK_MAJOR) == \
+            np.ravel_multi_index((blk, l, kv, slot, h, d, b), (NB, L, 2, BS, H, D, e))
+
+
+def dict_gather_block_major(pool, L, H, D, e, BS, NB, bt, n):
+    names = {}
+    it = iter(pool.tolist())
+    for key in itertools.product(range(NB), range(L), range(2), range(BS), range(H), range(D), range(e)):
+        names[key] = next(it)
+    out = [names[(bt[t // BS], l, kv, t % BS, h, d, b)]
+           for l, kv, t, h, d, b in itertools.product(range(L), range(2), range(n), range(H), range(D), range(e))]
+    return np.asarray(out, dtype=np.uint8)
+
+
+def test_block_major_gather_brute_force_and_numpy():
+    rng = np.random.default_rng(4)
+    cases = 0
+    for NB, BS in [(3, 1), (4, 2), (3, 3)]:
+        for L, H, D, e in [(1, 1, 1, 1), (2, 1, 2, 1), (2, 2, 1, 2)]:
+            pool = rng.integers(0, 256, size=NB * L * 2 * BS * H * D * e, dtype=np.uint8)
+            for nb in range(0, NB + 1):
+                for bt in itertools.permutations(range(NB), nb):
+                    for n in range((nb - 1) * BS + 1 if nb else 0, nb * BS + 1):
+                        got = orc.gather(pool, L, H, D, e, BS, NB, bt, n, layout=orc.BLOCK_MAJOR)
+                        assert np.array_equal(got, dict_gather_block_major(pool, L, H, D, e, BS, NB, bt, n))
+                        if nb:
+                            v = pool.reshape(NB, L, 2, BS, H * D * e)[np.asarray(bt)]          # [nb][L][2][BS][row]
+                            want = v.transpose(1, 2, 0, 3, 4).reshape(L, 2, nb * BS, -1)[:, :, :n].reshape(-1)
+                            assert np.array_equal(got, want)
+                        cases += 1
+    assert cases > 500
+
+
+def test_block_major_scatter_round_trip_and_pool_object():
+    L, H, D, e, BS, NB = 2, 2, 4, 2, 4, 10
+    rng = np.random.default_rng(6)
+    p = orc.OrcPool(L, H, D, e, BS, NB, 1 << 20, initial_free_order=rng.permutation(NB), layout=orc.BLOCK_MAJOR)
+    p.data[:] = fill_bytes(6, 0, p.data.size)
+    p.admit(1, 13)
+    tbl = p.info(1)[1]["blocks"]
+    want = orc.gather(p.data, L, H, D, e, BS, NB, tbl, 13, layout=orc.BLOCK_MAJOR).copy()
+    before = p.data.copy()
+    p.suspend_to_host([1])
+    assert np.array_equal(p.info(1)[1]["image"], want) and np.array_equal(p.data, before)
+    p.data.reshape(NB, -1)[p.free_queue()] ^= 0xFF
+    mid = p.data.copy()
+    p.resume_from_host([1])
+    new = p.info(1)[1]["blocks"]
+    assert np.array_equal(orc.gather(p.data, L, H, D, e, BS, NB, new, 13, layout=orc.BLOCK_MAJOR), want)
+    # only the valid slots of the destination blocks changed
+    mask = np.zeros((NB, L, 2, BS, H * D * e), dtype=bool)
+    for t in range(13):
+        mask[new[t // BS], :, :, t % BS] = True
+    assert not ((p.data != mid).reshape(mask.shape) & ~mask).any()
