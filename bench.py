@@ -332,12 +332,13 @@ def run_ours(args):
         view[i:i + step_elems].normal_(generator=gen)
     torch.cuda.synchronize()
 
-    route = {"staged": kvr.ROUTE_STAGED, "mapped": kvr.ROUTE_MAPPED}[args.route]
+    route = {"staged": kvr.ROUTE_STAGED, "mapped": kvr.ROUTE_MAPPED, "dma2d": kvr.ROUTE_DMA2D}[args.route]
+    layout = {"layer": kvr.LAYER_MAJOR, "block": kvr.BLOCK_MAJOR}[args.layout]
     kernel = {"warp": kvr.KERNEL_WARP, "bulk": kvr.KERNEL_BULK}[args.kernel]
     pool = kvr.Pool(*w.geom, w.num_blocks, host_cap, initial_free_order=free_order(seed, w.num_blocks),
                     device=local, device_pool=dev_pool.data_ptr(), route=route, kernel=kernel,
                     chunk_bytes=args.chunk_mib << 20, staging_slots=args.slots, max_ctas=args.max_ctas,
-                    flags=kvr.PROFILE)
+                    flags=kvr.PROFILE, layout=layout)
 
     # live set: the batch and the fillers, admitted in a seeded interleaved order (fragmented placement)
     ids = list(range(len(lens)))
@@ -478,7 +479,7 @@ def run_ours(args):
             "config": {"workload": w.name, "geometry": dict(zip(("layers", "kv_heads", "head_dim", "dtype_bytes", "block_size"), w.geom)),
                        "num_blocks": w.num_blocks, "requests_requested": requested, "requests_run": len(ids),
                        "tokens": int(lens.sum()), "payload_bytes_per_direction": payload,
-                       "occupancy_before_suspend": occupancy, "route": args.route, "kernel": args.kernel,
+                       "occupancy_before_suspend": occupancy, "route": args.route, "layout": args.layout, "kernel": args.kernel,
                        "chunk_mib": args.chunk_mib, "staging_slots": args.slots, "seed": seed,
                        "l2": "inputs (tens of GiB) are far larger than L2; no flush needed",
                        "timing": "value: CUDA events, first enqueued work to last byte landed, summed over the two batched moves of each step; e2e: host clock around the K steps"},
@@ -503,7 +504,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama3_8b", choices=list(CONFIGS))
-    ap.add_argument("--route", default="staged", choices=["staged", "mapped"])
+    ap.add_argument("--route", default="staged", choices=["staged", "mapped", "dma2d"])
+    ap.add_argument("--layout", default="layer", choices=["layer", "block"], help="pool layout: layer-major or block-major")
     ap.add_argument("--kernel", default="bulk", choices=["warp", "bulk"])
     ap.add_argument("--chunk-mib", type=int, default=512)
     ap.add_argument("--slots", type=int, default=2)

@@ -17,6 +17,8 @@
  * Layouts (the paper leaves them open; they are fixed here):
  *   pool  : bytes [layers][2][num_blocks][block_size][kv_heads][head_dim][dtype_bytes]
  *           plane 0 = K, plane 1 = V; one (layer, plane, block) tile is contiguous
+ *           (KVR_LAYER_MAJOR, the default); or, with KVR_BLOCK_MAJOR,
+ *           bytes [num_blocks][layers][2][block_size][kv_heads][head_dim][dtype_bytes]
  *   image : bytes [layers][2][n_tokens][kv_heads][head_dim][dtype_bytes]
  *           exactly n_tokens * kvr_bytes_per_token() bytes, valid tokens only
  * Bookkeeping rules (also fixed here): the free queue is FIFO (allocate from
@@ -80,8 +82,12 @@ enum {
 
 #define KVR_ROUTE_STAGED 1           /* kernel <-> HBM staging ring <-> chunked cudaMemcpyAsync */
 #define KVR_ROUTE_MAPPED 2           /* kernel reads / writes the pinned arena directly over the host link */
+#define KVR_ROUTE_DMA2D 3            /* no kernel: one strided cudaMemcpy2DAsync per block, pool <-> arena */
 #define KVR_KERNEL_WARP 1            /* one warp per tile, 16-byte loads and stores */
 #define KVR_KERNEL_BULK 2            /* bulk async copies through a shared-memory ring */
+
+#define KVR_LAYER_MAJOR 0
+#define KVR_BLOCK_MAJOR 1
 
 #define KVR_ALL UINT64_MAX
 
@@ -100,7 +106,7 @@ typedef struct {
   int32_t kernel;                    /* KVR_KERNEL_*; 0 = KVR_KERNEL_BULK */
   int32_t max_ctas;                  /* cap on the movers' grid (0 = fill the GPU) */
   uint32_t flags;                    /* KVR_METADATA_ONLY | KVR_PROFILE */
-  uint32_t reserved;
+  int32_t layout;                    /* KVR_LAYER_MAJOR (0) or KVR_BLOCK_MAJOR */
   void *device_pool;                 /* DEVICE pointer to num_blocks*block_size*bytes_per_token bytes,
                                         256-byte aligned, or NULL: the library allocates and frees it */
   void *host_arena;                  /* page-locked HOST pointer to host_capacity_bytes bytes, 4096-byte
@@ -233,6 +239,7 @@ kvr_status kvr_import_from_device(kvr_pool *pool, const uint64_t *req, int32_t n
  * the array needs clearing: each call overwrites what it uses.
  */
 #define KVR_NOALLOC_MAX_BLOCKS 65536
+/* (the pool is taken to be KVR_LAYER_MAJOR) */
 kvr_status kvr_gather_noalloc(const void *device_pool, const kvr_geometry *g, int32_t num_blocks,
                               const int32_t *block_table, int32_t nb, int64_t n_tokens,
                               void *dst_device, void *stream);

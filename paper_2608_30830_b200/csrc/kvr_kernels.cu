@@ -68,7 +68,7 @@ __device__ __forceinline__ Tile locate(const MoveArgs &a, const long long *cum, 
   long long valid = sg.n_tokens - first_tok;
   if (valid > a.block_size) valid = a.block_size;
   Tile t;
-  t.pool_ptr = a.pool + plane * a.plane_stride + (long long)blk * a.tile_bytes;
+  t.pool_ptr = a.pool + plane * a.plane_stride + (long long)blk * a.block_stride;
   t.lin_ptr = sg.img + (plane * sg.n_tokens + first_tok) * a.row_bytes;
   t.bytes = (int)valid * a.row_bytes;
   return t;

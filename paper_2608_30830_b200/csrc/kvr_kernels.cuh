@@ -27,7 +27,8 @@ struct MoveArgs {
   int nsegs;
   long long total_tiles; // sum of tile_count
   char *pool;            // DEVICE: paged pool base
-  long long plane_stride;// bytes of one (layer, plane): num_blocks * tile_bytes
+  long long plane_stride;// bytes from one (layer, plane) to the next, for a fixed block
+  long long block_stride;// bytes from one block to the next, for a fixed plane
   int tile_bytes;        // block_size * row_bytes
   int row_bytes;         // kv_heads * head_dim * dtype_bytes (multiple of 16)
   int block_size;

@@ -121,7 +121,7 @@ struct kvr_pool {
   bool meta_only = false, profile = false;
   uint64_t bpt = 0;
   int row = 0, tile_bytes = 0;
-  long long plane_stride = 0;
+  long long plane_stride = 0, block_stride = 0;
   int32_t NB = 0, BS = 0, planes = 0;
 
   FreeQueue fq;
@@ -358,7 +358,7 @@ void plan_direct(kvr_pool *p, const std::vector<Item> &items, char *lin_base, co
 kvr_status launch(kvr_pool *p, bool gather, const Seg *segs_dev, const Chunk &c, cudaStream_t s, Op &op) {
   MoveArgs a{};
   a.segs = segs_dev + c.seg_begin; a.nsegs = c.nsegs; a.total_tiles = c.tiles;
-  a.pool = p->d_pool; a.plane_stride = p->plane_stride; a.tile_bytes = p->tile_bytes;
+  a.pool = p->d_pool; a.plane_stride = p->plane_stride; a.block_stride = p->block_stride; a.tile_bytes = p->tile_bytes;
   a.row_bytes = p->row; a.block_size = p->BS; a.status = p->status_word;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   if (p->profile) {
@@ -376,6 +376,63 @@ kvr_status launch(kvr_pool *p, bool gather, const Seg *segs_dev, const Chunk &c,
   return KVR_OK;
 }
 
+void register_op(kvr_pool *p, Op &op, std::vector<Item> &items, const std::vector<int> &req_chunk, int kind,
+                 Clock::time_point t_call, uint64_t *out_seq) {
+  op.host_ms = ms_since(t_call);
+  for (size_t i = 0; i < items.size(); ++i) {
+    op.reqs.push_back({items[i].id, req_chunk[i]});
+    if (items[i].r) {
+      items[i].r->pending_op = op.seq;
+      items[i].r->pending_kind = kind == OP_SUSPEND ? KVR_SUSPENDING : kind == OP_RESUME ? KVR_RESUMING : 0;
+      items[i].r->has_latency = false;
+    }
+  }
+  *out_seq = op.seq;
+  p->ops.emplace(op.seq, std::move(op));
+}
+
+// Strided-copy route: no kernel and no staging.  For every block, one cudaMemcpy2DAsync moves its 2L tiles
+// (rows of `width` valid bytes, `plane_stride` apart in the pool, one image plane apart in the arena).
+kvr_status enqueue_dma2d(kvr_pool *p, Op &op, std::vector<Item> &items, bool to_linear, uint64_t block_tag,
+                         const std::vector<uint64_t> &arena_waits, Clock::time_point t_call, uint64_t *out_seq) {
+  cudaStream_t c = to_linear ? p->s_d2h : p->s_h2d;
+  kvr_status s;
+  CU(cudaEventRecord(op.start, c));
+  for (auto &it : items)
+    if (it.r && it.r->pending_op && (s = stream_after(p, c, it.r->pending_op, false))) return s;
+  if (!to_linear && (s = stream_after(p, c, block_tag, true))) return s;
+  for (uint64_t w : arena_waits) if ((s = stream_after(p, c, w, true))) return s;
+  std::vector<int> req_chunk(items.size(), -1);
+  for (size_t i = 0; i < items.size(); ++i) {
+    const Item &it = items[i];
+    if (!it.nb) continue;
+    const size_t img_pitch = (size_t)it.n_tokens * p->row;
+    for (int32_t b = 0; b < it.nb; ++b) {
+      long long valid = it.n_tokens - (long long)b * p->BS;
+      if (valid > p->BS) valid = p->BS;
+      const size_t width = (size_t)valid * p->row;
+      char *pool_ptr = p->d_pool + (long long)it.blocks[b] * p->block_stride;
+      char *img_ptr = p->h_arena + it.lin_off + (size_t)b * p->BS * p->row;
+      if (to_linear) {
+        CU(cudaMemcpy2DAsync(img_ptr, img_pitch, pool_ptr, (size_t)p->plane_stride, width, (size_t)p->planes, cudaMemcpyDeviceToHost, c));
+        p->st.d2h_copies++; p->st.d2h_bytes += width * p->planes;
+      } else {
+        CU(cudaMemcpy2DAsync(pool_ptr, (size_t)p->plane_stride, img_ptr, img_pitch, width, (size_t)p->planes, cudaMemcpyHostToDevice, c));
+        p->st.h2d_copies++; p->st.h2d_bytes += width * p->planes;
+      }
+    }
+    cudaEvent_t cd;
+    if ((s = get_event(p, &cd))) return s;
+    CU(cudaEventRecord(cd, c));
+    req_chunk[i] = (int)op.chunk_done.size();
+    op.chunk_done.push_back(cd);
+  }
+  CU(cudaEventRecord(op.read_done, c));
+  CU(cudaEventRecord(op.done, c));
+  register_op(p, op, items, req_chunk, op.kind, t_call, out_seq);
+  return KVR_OK;
+}
+
 // Build and upload the descriptors of a move, then enqueue it.  `to_linear` = gather direction.
 // route: KVR_ROUTE_STAGED, KVR_ROUTE_MAPPED, or 0 for a caller-supplied device buffer (lin_dev).
 kvr_status enqueue(kvr_pool *p, int kind, std::vector<Item> &items, int route, char *lin_dev,
@@ -389,6 +446,8 @@ kvr_status enqueue(kvr_pool *p, int kind, std::vector<Item> &items, int route, c
   op.seq = p->next_seq++;
   op.kind = kind;
   if ((s = get_event(p, &op.start)) || (s = get_event(p, &op.read_done)) || (s = get_event(p, &op.done))) return s;
+
+  if (route == KVR_ROUTE_DMA2D) return enqueue_dma2d(p, op, items, to_linear, block_tag, arena_waits, t_call, out_seq);
 
   // plan with table addresses relative to the descriptor buffer, then size the buffer exactly:
   // [block tables][segments]
@@ -486,17 +545,7 @@ kvr_status enqueue(kvr_pool *p, int kind, std::vector<Item> &items, int route, c
   }
   CU(cudaEventRecord(op.done, last));
 
-  op.host_ms = ms_since(t_call);
-  for (size_t i = 0; i < items.size(); ++i) {
-    op.reqs.push_back({items[i].id, pl.req_chunk[i]});
-    if (items[i].r) {
-      items[i].r->pending_op = op.seq;
-      items[i].r->pending_kind = kind == OP_SUSPEND ? KVR_SUSPENDING : kind == OP_RESUME ? KVR_RESUMING : 0;
-      items[i].r->has_latency = false;
-    }
-  }
-  *out_seq = op.seq;
-  p->ops.emplace(op.seq, std::move(op));
+  register_op(p, op, items, pl.req_chunk, kind, t_call, out_seq);
   return KVR_OK;
 }
 
@@ -540,6 +589,9 @@ kvr_status create_engine(kvr_pool *p) {
   CU(cudaGetDeviceProperties(&prop, c.device));
   p->device = c.device;
   p->sm_count = prop.multiProcessorCount;
+  if (c.route == KVR_ROUTE_DMA2D && (size_t)p->plane_stride > prop.memPitch)
+    return fail(KVR_ERR_GEOMETRY, "strided-copy route: plane stride %lld exceeds the device's copy pitch limit %zu "
+                "(use the block-major layout or another route)", p->plane_stride, prop.memPitch);
   const uint64_t pool_bytes = (uint64_t)p->NB * p->BS * p->bpt;
   if (c.device_pool) p->d_pool = (char *)c.device_pool;
   else {
@@ -631,7 +683,8 @@ kvr_status kvr_pool_create(const kvr_config *cfg, kvr_pool **out) {
   if (!p->cfg.route) p->cfg.route = KVR_ROUTE_STAGED;
   if (!p->cfg.kernel) p->cfg.kernel = KVR_KERNEL_BULK;
   kvr_status bad = KVR_OK;
-  if (p->cfg.route != KVR_ROUTE_STAGED && p->cfg.route != KVR_ROUTE_MAPPED) bad = fail(KVR_ERR_INVALID_ARG, "unknown route");
+  if (p->cfg.route != KVR_ROUTE_STAGED && p->cfg.route != KVR_ROUTE_MAPPED && p->cfg.route != KVR_ROUTE_DMA2D) bad = fail(KVR_ERR_INVALID_ARG, "unknown route");
+  else if (p->cfg.layout != KVR_LAYER_MAJOR && p->cfg.layout != KVR_BLOCK_MAJOR) bad = fail(KVR_ERR_INVALID_ARG, "unknown layout");
   else if (p->cfg.kernel != KVR_KERNEL_WARP && p->cfg.kernel != KVR_KERNEL_BULK) bad = fail(KVR_ERR_INVALID_ARG, "unknown kernel");
   else if (p->cfg.chunk_bytes % 4096 || p->cfg.chunk_bytes < tile) bad = fail(KVR_ERR_INVALID_ARG, "chunk_bytes must be a multiple of 4096 and hold one tile");
   else if (p->cfg.staging_slots < 2 || p->cfg.staging_slots > 64) bad = fail(KVR_ERR_INVALID_ARG, "staging_slots must be in [2, 64]");
@@ -649,7 +702,8 @@ kvr_status kvr_pool_create(const kvr_config *cfg, kvr_pool **out) {
   p->profile = cfg->flags & KVR_PROFILE;
   p->bpt = bpt; p->row = (int)row; p->tile_bytes = (int)tile;
   p->NB = cfg->num_blocks; p->BS = cfg->g.block_size; p->planes = 2 * cfg->g.layers;
-  p->plane_stride = (long long)p->NB * p->tile_bytes;
+  if (p->cfg.layout == KVR_BLOCK_MAJOR) { p->plane_stride = p->tile_bytes; p->block_stride = (long long)p->planes * p->tile_bytes; }
+  else { p->plane_stride = (long long)p->NB * p->tile_bytes; p->block_stride = p->tile_bytes; }
   p->fq.init(p->NB, cfg->initial_free_order);
   p->arena.init(cfg->host_capacity_bytes);
   p->cfg.initial_free_order = nullptr;

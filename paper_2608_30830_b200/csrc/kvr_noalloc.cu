@@ -106,7 +106,8 @@ extern "C" kvr_status kvr_gather_noalloc(const void *device_pool, const kvr_geom
   a.total_tiles = seg.tile_count;
   a.pool = static_cast<char *>(const_cast<void *>(device_pool));
   a.tile_bytes = row * g->block_size;
-  a.plane_stride = (long long)num_blocks * a.tile_bytes;
+  a.plane_stride = (long long)num_blocks * a.tile_bytes;   // layer-major pool
+  a.block_stride = a.tile_bytes;
   a.row_bytes = row;
   a.block_size = g->block_size;
   a.status = nullptr;               // the warp mover has no bounded waits and never writes it

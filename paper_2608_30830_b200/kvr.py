@@ -12,7 +12,8 @@ ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM = -5, -6, -7
 ACTIVE, RETAINED, SUSPENDING, HOST, RESUMING, EXPIRED = 0, 1, 2, 3, 4, 5
 SYNC = 1
 METADATA_ONLY, PROFILE = 1, 2
-ROUTE_STAGED, ROUTE_MAPPED = 1, 2
+ROUTE_STAGED, ROUTE_MAPPED, ROUTE_DMA2D = 1, 2, 3
+LAYER_MAJOR, BLOCK_MAJOR = 0, 1
 KERNEL_WARP, KERNEL_BULK = 1, 2
 ALL = 2**64 - 1
 
@@ -31,7 +32,7 @@ class Config(C.Structure):
     _fields_ = [("g", Geometry), ("num_blocks", C.c_int32), ("device", C.c_int32),
                 ("host_capacity_bytes", C.c_uint64), ("chunk_bytes", C.c_uint64),
                 ("staging_slots", C.c_int32), ("route", C.c_int32), ("kernel", C.c_int32),
-                ("max_ctas", C.c_int32), ("flags", C.c_uint32), ("reserved", C.c_uint32),
+                ("max_ctas", C.c_int32), ("flags", C.c_uint32), ("layout", C.c_int32),
                 ("device_pool", C.c_void_p), ("host_arena", C.c_void_p),
                 ("initial_free_order", C.POINTER(C.c_int32))]
 
@@ -165,14 +166,15 @@ class Pool:
 
     def __init__(self, layers, kv_heads, head_dim, dtype_bytes, block_size, num_blocks, host_capacity_bytes,
                  initial_free_order=None, device=0, chunk_bytes=0, staging_slots=0, route=0, kernel=0,
-                 max_ctas=0, flags=0, device_pool=None, host_arena=None):
+                 max_ctas=0, flags=0, device_pool=None, host_arena=None, layout=0):
         self.geom = (layers, kv_heads, head_dim, dtype_bytes, block_size)
         self.NB = num_blocks
         cfg = Config()
         cfg.g = Geometry(*self.geom)
         cfg.num_blocks, cfg.device = num_blocks, device
         cfg.host_capacity_bytes, cfg.chunk_bytes, cfg.staging_slots = host_capacity_bytes, chunk_bytes, staging_slots
-        cfg.route, cfg.kernel, cfg.max_ctas, cfg.flags = route, kernel, max_ctas, flags
+        cfg.route, cfg.kernel, cfg.max_ctas, cfg.flags, cfg.layout = route, kernel, max_ctas, flags, layout
+        self.layout = layout
         cfg.device_pool = device_pool
         cfg.host_arena = host_arena
         order = None

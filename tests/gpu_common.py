@@ -11,18 +11,19 @@ from paper_2608_30830_b200 import kvr
 class Twin:
     """Oracle pool + library pool with identical geometry, free order and initial pool bytes."""
 
-    def __init__(self, geom, NB, host_cap, seed=0, order=None, **lib_kw):
+    def __init__(self, geom, NB, host_cap, seed=0, order=None, layout=0, **lib_kw):
         L, H, D, e, BS = geom
         self.geom, self.NB = geom, NB
         if order is None:
             order = np.random.default_rng(seed).permutation(NB).astype(np.int32)
-        self.o = orc.OrcPool(*geom, NB, host_cap, initial_free_order=order, with_data=True)
+        self.layout = layout
+        self.o = orc.OrcPool(*geom, NB, host_cap, initial_free_order=order, with_data=True, layout=layout)
         nbytes = self.o.data.size
         self.o.data[:] = fill_bytes(seed, 0, nbytes, e)
         self.dev = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
         self.dev.copy_(torch.from_numpy(self.o.data))
         torch.cuda.synchronize()
-        self.g = kvr.Pool(*geom, NB, host_cap, initial_free_order=order, device_pool=self.dev.data_ptr(), **lib_kw)
+        self.g = kvr.Pool(*geom, NB, host_cap, initial_free_order=order, device_pool=self.dev.data_ptr(), layout=layout, **lib_kw)
 
     def pool_bytes(self):
         assert self.g.wait() == kvr.OK

@@ -21,6 +21,10 @@ MODES = [
     pytest.param(dict(route=kvr.ROUTE_STAGED, kernel=kvr.KERNEL_BULK), id="staged-bulk"),
     pytest.param(dict(route=kvr.ROUTE_MAPPED, kernel=kvr.KERNEL_WARP), id="mapped-warp"),
     pytest.param(dict(route=kvr.ROUTE_MAPPED, kernel=kvr.KERNEL_BULK), id="mapped-bulk"),
+    pytest.param(dict(route=kvr.ROUTE_STAGED, kernel=kvr.KERNEL_BULK, layout=kvr.BLOCK_MAJOR), id="staged-bulk-blockmajor"),
+    pytest.param(dict(route=kvr.ROUTE_MAPPED, kernel=kvr.KERNEL_WARP, layout=kvr.BLOCK_MAJOR), id="mapped-warp-blockmajor"),
+    pytest.param(dict(route=kvr.ROUTE_DMA2D), id="dma2d"),
+    pytest.param(dict(route=kvr.ROUTE_DMA2D, layout=kvr.BLOCK_MAJOR), id="dma2d-blockmajor"),
 ]
 SMALL = (3, 2, 16, 2, 8)          # L, H, D, e, BS: 64-byte rows, 512-byte tiles, 384 bytes per token
 LENGTHS = [0, 1, 7, 8, 9, 64, 67, 200, 3, 16]
@@ -44,12 +48,15 @@ def test_suspend_then_resume_small(mode):
     t.assert_same_pool()                                  # only valid slots of the new blocks changed
     check_invariants(t.g, ids)
     s = t.g.stats()
-    assert s["gather_launches"] >= 1 and s["scatter_launches"] >= 1
-    assert s["gather_bytes"] == s["scatter_bytes"] == sum(LENGTHS) * 384
+    if mode.get("route") == kvr.ROUTE_DMA2D:
+        assert s["gather_launches"] == s["scatter_launches"] == 0 and s["d2h_bytes"] == s["h2d_bytes"] == sum(LENGTHS) * 384
+    else:
+        assert s["gather_launches"] >= 1 and s["scatter_launches"] >= 1
+        assert s["gather_bytes"] == s["scatter_bytes"] == sum(LENGTHS) * 384
     t.close()
 
 
-@pytest.mark.parametrize("mode", MODES[:2])
+@pytest.mark.parametrize("mode", MODES[:2] + MODES[4:5])
 def test_export_import_kernels_alone(mode):
     """gather and scatter kernels HBM to HBM, against the oracle's per-element loops."""
     t = Twin(SMALL, 96, 0, seed=2, **mode)
@@ -65,7 +72,7 @@ def test_export_import_kernels_alone(mode):
     assert st == kvr.OK, kvr.last_error()
     host = buf.cpu().numpy()
     for rid, n, off in zip(ids, LENGTHS, offs):
-        want = orc.gather(t.o.data, L, H, D, e, BS, t.NB, tables[rid], n)
+        want = orc.gather(t.o.data, L, H, D, e, BS, t.NB, tables[rid], n, layout=t.layout)
         assert off % 256 == 0 and np.array_equal(host[int(off):int(off) + want.size], want)
     # scatter new content back through the same tables
     new = np.random.default_rng(5).integers(0, 256, size=cap, dtype=np.uint8)
@@ -74,7 +81,7 @@ def test_export_import_kernels_alone(mode):
     st, offs2 = t.g.import_from_device(ids, buf.data_ptr(), cap, kvr.SYNC)
     assert st == kvr.OK and offs2.tolist() == offs.tolist()
     for rid, n, off in zip(ids, LENGTHS, offs):
-        orc.scatter(t.o.data, new[int(off):int(off) + n * 384], L, H, D, e, BS, t.NB, tables[rid], n)
+        orc.scatter(t.o.data, new[int(off):int(off) + n * 384], L, H, D, e, BS, t.NB, tables[rid], n, layout=t.layout)
     t.assert_same_pool()
     assert t.g.export_to_device(ids, buf.data_ptr(), 100)[0] == kvr.ERR_INVALID_ARG
     t.close()
@@ -178,6 +185,31 @@ def test_transient_states_and_latency():
     assert t.g.wait(99) == kvr.ERR_UNKNOWN_REQUEST
     t.assert_same_pool()
     t.close()
+
+
+def test_fp8_sized_elements():
+    """dtype_bytes = 1 (fp8 KV): 1 KiB rows; the movers are byte-exact whatever the element type."""
+    geom = (4, 8, 128, 1, 16)
+    t = Twin(geom, 96, 1 << 22, seed=12, chunk_bytes=1 << 16)
+    lens = [100, 257, 16, 1]
+    for rid, n in enumerate(lens):
+        assert t.both("admit", rid, n)[1][0] == kvr.OK
+    assert kvr.bytes_per_token(4, 8, 128, 1) == 8192
+    ids = list(range(len(lens)))
+    a, b = t.both("suspend_to_host", ids)
+    assert a == b
+    t.assert_same_images(ids)
+    a, b = t.both("resume_from_host", ids)
+    assert a == b
+    t.assert_same_pool()
+    t.close()
+
+
+def test_strided_copy_route_rejects_an_oversized_pitch():
+    # layer-major plane stride = num_blocks x tile; beyond the device's copy pitch limit the route is refused
+    with pytest.raises(kvr.KvrError) as e:
+        kvr.Pool(1, 8, 128, 2, 16, 1 << 17, 0, route=kvr.ROUTE_DMA2D, device_pool=256)
+    assert e.value.status == kvr.ERR_GEOMETRY and "pitch" in str(e.value)
 
 
 def test_wait_is_bounded():
