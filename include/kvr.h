@@ -276,6 +276,29 @@ kvr_status kvr_wait(kvr_pool *pool, uint64_t req_or_all, int64_t timeout_ms);
 kvr_status kvr_read_load(const void *device_buf, uint64_t bytes, int32_t launches, void *device_sink, void *stream);
 
 kvr_status kvr_pool_stats(kvr_pool *pool, kvr_stats *out);
+
+/*
+ * The policy that decides when the moves above happen (host code, no GPU work; all times in seconds, costs in
+ * GPU-seconds).  kvr_prices is the platform's calibrated price vector (Section 3.2): alpha1 = HBM holding cost per
+ * second, beta2 = host-resume cost, beta3 = recomputation cost; valid iff alpha1 > 0 and beta3 > beta2 >= 0.
+ */
+typedef struct { double alpha1, beta2, beta3; } kvr_prices;
+/* Eq. 2: t_1 = beta2 / alpha1 (HBM vs host break-even), t* = beta3 / alpha1 (HBM vs discard). */
+kvr_status kvr_policy_break_evens(const kvr_prices *p, double *t1, double *t_star);
+/* Eq. 3: lambda_crit = c2 / w_ref; alpha2 = max(0, lambda - lambda_crit) * beta3 / c2; t2 = (beta3 - beta2) / alpha2,
+ * +infinity at or below lambda_crit.  c2 = contexts that fit in the host tier.  Either out pointer may be NULL. */
+kvr_status kvr_policy_host_ttl(const kvr_prices *p, double lambda, double c2, double w_ref, double *alpha2, double *t2);
+/* Measured-cost replay (Appendix D): contexts arrive at arrive[i] (non-decreasing) and wait wait[i]; each is
+ * admitted iff one of c2 slots is free, residents are never displaced; a slot is held until the resume or until
+ * ttl after arrival (one-shot timer, +infinity = host-retain).  A resume that finds its copy costs beta2, any other
+ * beta3.  Outputs: mean cost per request and the fraction resumed from the host copy. */
+kvr_status kvr_policy_replay(const kvr_prices *p, const double *arrive, const double *wait, int64_t n, int64_t c2,
+                             double ttl, double *mean_cost, double *from_host);
+/* Controller (Section 3.4): replay a calibration sample under host-retain and under cpu_ttl(lambda), report both
+ * costs and the timer, and set *use_ttl to 1 iff expiration is strictly cheaper.  Out pointers may be NULL. */
+kvr_status kvr_policy_select(const kvr_prices *p, const double *arrive, const double *wait, int64_t n, double lambda,
+                             int64_t c2, double w_ref, int32_t *use_ttl, double *cost_retain, double *cost_ttl, double *t2);
+
 /* copies the free queue, head first, into out (cap entries, may be NULL); returns its length */
 int64_t kvr_free_queue(kvr_pool *pool, int32_t *out, int64_t cap);
 /* the DEVICE pool pointer and the HOST arena pointer in use (caller's or the library's) */

@@ -7,5 +7,5 @@ the CPU oracle's tests and the CUDA library's tests may take inputs from it.
 """
 from .gen import (  # noqa: F401
     CONFIGS, Workload, bf16_normal_bits, context_lengths, event_trace, fill_bytes,
-    free_order, occupancy_fillers, wait_mixture,
+    free_order, occupancy_fillers, paper_wait_family, poisson_arrivals, wait_mixture,
 )

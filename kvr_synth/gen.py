@@ -132,3 +132,27 @@ def event_trace(n_requests, seed, arrival_rate, t_offload, t_expire):
         ev.append((t0 + w, len(ev), "resume", i))
     ev.sort()
     return ev, waits
+
+
+def paper_wait_family(name, n, seed, mean_s=1800.0):
+    """Waits of the paper's three replay families, each with mean `mean_s`: 'lognormal' (sigma 1),
+    'exponential', 'mixture' (half exponential with mean 60 s, half lognormal with sigma 0.7 and mean 3,540 s)."""
+    r = _rng(seed, 6)
+    if name == "lognormal":
+        sigma = 1.0
+        return np.exp(np.log(mean_s) - sigma * sigma / 2 + sigma * r.standard_normal(n))
+    if name == "exponential":
+        return r.exponential(mean_s, size=n)
+    if name == "mixture":
+        scale = mean_s / 1800.0
+        pick = r.random(n) < 0.5
+        short = r.exponential(60.0 * scale, size=n)
+        sigma = 0.7
+        long_ = np.exp(np.log(3540.0 * scale) - sigma * sigma / 2 + sigma * r.standard_normal(n))
+        return np.where(pick, short, long_)
+    raise ValueError(name)
+
+
+def poisson_arrivals(n, rate, seed):
+    """Arrival times of n requests of a Poisson process of the given rate."""
+    return np.cumsum(_rng(seed, 7).exponential(1.0 / rate, size=n))

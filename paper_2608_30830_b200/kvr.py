@@ -37,6 +37,10 @@ class Config(C.Structure):
                 ("initial_free_order", C.POINTER(C.c_int32))]
 
 
+class Prices(C.Structure):
+    _fields_ = [("alpha1", C.c_double), ("beta2", C.c_double), ("beta3", C.c_double)]
+
+
 class Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("blocks_total", "blocks_free", "blocks_active", "blocks_pinned")] + \
                [(n, C.c_uint64) for n in ("host_capacity", "host_used", "host_largest_hole")] + \
@@ -59,6 +63,7 @@ EXPORTS = [
     "kvr_resume_from_host_into", "kvr_export_to_device", "kvr_import_from_device", "kvr_request_info",
     "kvr_request_latency", "kvr_wait", "kvr_pool_stats", "kvr_free_queue", "kvr_pool_device_ptr",
     "kvr_pool_host_arena", "kvr_last_error", "kvr_gather_noalloc", "kvr_read_load",
+    "kvr_policy_break_evens", "kvr_policy_host_ttl", "kvr_policy_replay", "kvr_policy_select",
 ]
 
 _lib = None
@@ -118,6 +123,15 @@ def lib():
     L.kvr_pool_host_arena.argtypes = [vp]
     L.kvr_last_error.restype = C.c_char_p
     L.kvr_last_error.argtypes = []
+    pd = C.POINTER(C.c_double)
+    L.kvr_policy_break_evens.restype = i32
+    L.kvr_policy_break_evens.argtypes = [C.POINTER(Prices), pd, pd]
+    L.kvr_policy_host_ttl.restype = i32
+    L.kvr_policy_host_ttl.argtypes = [C.POINTER(Prices), C.c_double, C.c_double, C.c_double, pd, pd]
+    L.kvr_policy_replay.restype = i32
+    L.kvr_policy_replay.argtypes = [C.POINTER(Prices), pd, pd, i64, i64, C.c_double, pd, pd]
+    L.kvr_policy_select.restype = i32
+    L.kvr_policy_select.argtypes = [C.POINTER(Prices), pd, pd, i64, C.c_double, i64, C.c_double, pi32, pd, pd, pd]
     L.kvr_read_load.restype = i32
     L.kvr_read_load.argtypes = [vp, u64, i32, vp, vp]
     L.kvr_gather_noalloc.restype = i32
@@ -133,6 +147,43 @@ def last_error():
 def bytes_per_token(layers, kv_heads, head_dim, dtype_bytes, block_size=16):
     g = Geometry(layers, kv_heads, head_dim, dtype_bytes, block_size)
     return int(lib().kvr_bytes_per_token(C.byref(g)))
+
+
+def _check(st):
+    if st != OK:
+        raise KvrError(st, last_error())
+
+
+def policy_break_evens(alpha1, beta2, beta3):
+    p, t1, ts = Prices(alpha1, beta2, beta3), C.c_double(), C.c_double()
+    _check(lib().kvr_policy_break_evens(C.byref(p), C.byref(t1), C.byref(ts)))
+    return t1.value, ts.value
+
+
+def policy_host_ttl(prices, lam, c2, w_ref):
+    p, a2, t2 = Prices(*prices), C.c_double(), C.c_double()
+    _check(lib().kvr_policy_host_ttl(C.byref(p), lam, c2, w_ref, C.byref(a2), C.byref(t2)))
+    return a2.value, t2.value
+
+
+def _f64p(a):
+    return a.ctypes.data_as(C.POINTER(C.c_double))
+
+
+def policy_replay(prices, arrive, wait, c2, ttl):
+    p, cost, frac = Prices(*prices), C.c_double(), C.c_double()
+    arrive, wait = np.ascontiguousarray(arrive, dtype=np.float64), np.ascontiguousarray(wait, dtype=np.float64)
+    _check(lib().kvr_policy_replay(C.byref(p), _f64p(arrive), _f64p(wait), len(arrive), c2, ttl, C.byref(cost), C.byref(frac)))
+    return cost.value, frac.value
+
+
+def policy_select(prices, arrive, wait, lam, c2, w_ref):
+    p = Prices(*prices)
+    use, cr, ct, t2 = C.c_int32(), C.c_double(), C.c_double(), C.c_double()
+    arrive, wait = np.ascontiguousarray(arrive, dtype=np.float64), np.ascontiguousarray(wait, dtype=np.float64)
+    _check(lib().kvr_policy_select(C.byref(p), _f64p(arrive), _f64p(wait), len(arrive), lam, c2, w_ref,
+                                   C.byref(use), C.byref(cr), C.byref(ct), C.byref(t2)))
+    return ("ttl" if use.value else "retain"), cr.value, ct.value, t2.value
 
 
 def read_load(device_buf, nbytes, launches, device_sink, stream=None):
