@@ -299,6 +299,50 @@ kvr_status kvr_policy_replay(const kvr_prices *p, const double *arrive, const do
 kvr_status kvr_policy_select(const kvr_prices *p, const double *arrive, const double *wait, int64_t n, double lambda,
                              int64_t c2, double w_ref, int32_t *use_ttl, double *cost_retain, double *cost_ttl, double *t2);
 
+/*
+ * Live controller (Section 3.4 and the live-controller rules of Appendix D), host code on top of the calls above.
+ * It keeps a clock the caller advances (seconds, never backwards).  At a suspension the context is pinned in HBM
+ * (kvr_retain_in_hbm) and, after hbm_grace_s (0 = at once: t_1 is about a second), moved to the host tier; under
+ * KVR_BRANCH_TTL it then gets a one-shot timer t_2(lambda) counted from the offload.  When the host tier is full,
+ * KVR_ADMIT_REPLAY discards the newcomer (residents are never displaced) and KVR_ADMIT_LIVE first discards the
+ * host copy that has been suspended longest.  gpu_cost accumulates Eq. 1: alpha1 x seconds spent pinned in HBM,
+ * beta2 per resume from the host copy, beta3 per resume that must recompute.
+ */
+typedef struct kvr_controller kvr_controller;
+#define KVR_BRANCH_RETAIN 0
+#define KVR_BRANCH_TTL 1
+#define KVR_ADMIT_REPLAY 0
+#define KVR_ADMIT_LIVE 1
+typedef struct {
+  kvr_prices prices;
+  double lambda;             /* offered rate of suspensions, per second */
+  double c2;                 /* contexts the host tier holds; <= 0: host capacity / mean_image_bytes */
+  double mean_image_bytes;
+  double w_ref;              /* reference wait, seconds */
+  double hbm_grace_s;
+  int32_t branch;            /* KVR_BRANCH_* (kvr_controller_calibrate overrides it) */
+  int32_t admission;         /* KVR_ADMIT_* */
+} kvr_controller_config;
+typedef struct {
+  int64_t suspended, offloaded, not_admitted, ttl_expired, evicted_lru;
+  int64_t resumed_host, resumed_hbm, recomputed, tracked;
+  double gpu_cost, t2;
+  int32_t branch, reserved;
+} kvr_controller_stats;
+kvr_status kvr_controller_create(kvr_pool *pool, const kvr_controller_config *cfg, kvr_controller **out);
+kvr_status kvr_controller_destroy(kvr_controller *c);
+/* replay the calibration sample under both branches and freeze the cheaper one (kvr_policy_select) */
+kvr_status kvr_controller_calibrate(kvr_controller *c, const double *arrive, const double *wait, int64_t n, int32_t *branch);
+/* the ACTIVE request `req` suspends at time now: KVR_OK (on the host), KVR_RESIDENT (pinned in HBM for the grace
+ * period), KVR_HOST_FULL (not admitted: discarded, it will recompute) */
+kvr_status kvr_controller_suspend(kvr_controller *c, uint64_t req, double now);
+/* fire every offload and expiry due by `now`; counts may be NULL */
+kvr_status kvr_controller_advance(kvr_controller *c, double now, int32_t *n_offloaded, int32_t *n_expired);
+/* the request resumes at time now: KVR_OK (restored from host), KVR_RESIDENT, KVR_RECOMPUTE (caller re-admits and
+ * prefills), KVR_HBM_FULL (nothing changed; free blocks and call again) */
+kvr_status kvr_controller_resume(kvr_controller *c, uint64_t req, double now);
+kvr_status kvr_controller_get_stats(kvr_controller *c, kvr_controller_stats *out);
+
 /* copies the free queue, head first, into out (cap entries, may be NULL); returns its length */
 int64_t kvr_free_queue(kvr_pool *pool, int32_t *out, int64_t cap);
 /* the DEVICE pool pointer and the HOST arena pointer in use (caller's or the library's) */

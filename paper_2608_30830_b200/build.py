@@ -6,7 +6,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 SO = os.path.join(PKG, "libkvr.so")
-SOURCES = ["kvr_kernels.cu", "kvr_lib.cu", "kvr_noalloc.cu", "kvr_policy.cpp"]
+SOURCES = ["kvr_kernels.cu", "kvr_lib.cu", "kvr_noalloc.cu", "kvr_policy.cpp", "kvr_controller.cpp"]
 DEPS = SOURCES + ["kvr_kernels.cuh", "kvr_meta.hpp", os.path.join("..", "..", "include", "kvr.h")]
 
 

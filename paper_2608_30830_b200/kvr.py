@@ -41,6 +41,17 @@ class Prices(C.Structure):
     _fields_ = [("alpha1", C.c_double), ("beta2", C.c_double), ("beta3", C.c_double)]
 
 
+class ControllerConfig(C.Structure):
+    _fields_ = [("prices", Prices), ("lambda_", C.c_double), ("c2", C.c_double), ("mean_image_bytes", C.c_double),
+                ("w_ref", C.c_double), ("hbm_grace_s", C.c_double), ("branch", C.c_int32), ("admission", C.c_int32)]
+
+
+class ControllerStats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("suspended", "offloaded", "not_admitted", "ttl_expired", "evicted_lru",
+                                         "resumed_host", "resumed_hbm", "recomputed", "tracked")] + \
+               [("gpu_cost", C.c_double), ("t2", C.c_double), ("branch", C.c_int32), ("reserved", C.c_int32)]
+
+
 class Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("blocks_total", "blocks_free", "blocks_active", "blocks_pinned")] + \
                [(n, C.c_uint64) for n in ("host_capacity", "host_used", "host_largest_hole")] + \
@@ -64,6 +75,8 @@ EXPORTS = [
     "kvr_request_latency", "kvr_wait", "kvr_pool_stats", "kvr_free_queue", "kvr_pool_device_ptr",
     "kvr_pool_host_arena", "kvr_last_error", "kvr_gather_noalloc", "kvr_read_load",
     "kvr_policy_break_evens", "kvr_policy_host_ttl", "kvr_policy_replay", "kvr_policy_select",
+    "kvr_controller_create", "kvr_controller_destroy", "kvr_controller_calibrate", "kvr_controller_suspend",
+    "kvr_controller_advance", "kvr_controller_resume", "kvr_controller_get_stats",
 ]
 
 _lib = None
@@ -132,6 +145,20 @@ def lib():
     L.kvr_policy_replay.argtypes = [C.POINTER(Prices), pd, pd, i64, i64, C.c_double, pd, pd]
     L.kvr_policy_select.restype = i32
     L.kvr_policy_select.argtypes = [C.POINTER(Prices), pd, pd, i64, C.c_double, i64, C.c_double, pi32, pd, pd, pd]
+    L.kvr_controller_create.restype = i32
+    L.kvr_controller_create.argtypes = [vp, C.POINTER(ControllerConfig), C.POINTER(vp)]
+    L.kvr_controller_destroy.restype = i32
+    L.kvr_controller_destroy.argtypes = [vp]
+    L.kvr_controller_calibrate.restype = i32
+    L.kvr_controller_calibrate.argtypes = [vp, pd, pd, i64, pi32]
+    L.kvr_controller_suspend.restype = i32
+    L.kvr_controller_suspend.argtypes = [vp, u64, C.c_double]
+    L.kvr_controller_advance.restype = i32
+    L.kvr_controller_advance.argtypes = [vp, C.c_double, pi32, pi32]
+    L.kvr_controller_resume.restype = i32
+    L.kvr_controller_resume.argtypes = [vp, u64, C.c_double]
+    L.kvr_controller_get_stats.restype = i32
+    L.kvr_controller_get_stats.argtypes = [vp, C.POINTER(ControllerStats)]
     L.kvr_read_load.restype = i32
     L.kvr_read_load.argtypes = [vp, u64, i32, vp, vp]
     L.kvr_gather_noalloc.restype = i32
@@ -184,6 +211,51 @@ def policy_select(prices, arrive, wait, lam, c2, w_ref):
     _check(lib().kvr_policy_select(C.byref(p), _f64p(arrive), _f64p(wait), len(arrive), lam, c2, w_ref,
                                    C.byref(use), C.byref(cr), C.byref(ct), C.byref(t2)))
     return ("ttl" if use.value else "retain"), cr.value, ct.value, t2.value
+
+
+BRANCH_RETAIN, BRANCH_TTL = 0, 1
+ADMIT_REPLAY, ADMIT_LIVE = 0, 1
+
+
+class Controller:
+    """kvr_controller handle over a Pool (which must outlive it)."""
+
+    def __init__(self, pool, prices, lam, w_ref, c2=0.0, mean_image_bytes=0.0, hbm_grace_s=0.0,
+                 branch=BRANCH_RETAIN, admission=ADMIT_REPLAY):
+        cfg = ControllerConfig(Prices(*prices), lam, c2, mean_image_bytes, w_ref, hbm_grace_s, branch, admission)
+        h = C.c_void_p()
+        _check(lib().kvr_controller_create(pool._h, C.byref(cfg), C.byref(h)))
+        self._h, self.pool = h, pool
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().kvr_controller_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
+
+    def calibrate(self, arrive, wait):
+        arrive, wait = np.ascontiguousarray(arrive, dtype=np.float64), np.ascontiguousarray(wait, dtype=np.float64)
+        b = C.c_int32()
+        _check(lib().kvr_controller_calibrate(self._h, _f64p(arrive), _f64p(wait), len(arrive), C.byref(b)))
+        return b.value
+
+    def suspend(self, rid, now):
+        return lib().kvr_controller_suspend(self._h, rid, now)
+
+    def advance(self, now):
+        a, b = C.c_int32(), C.c_int32()
+        st = lib().kvr_controller_advance(self._h, now, C.byref(a), C.byref(b))
+        return st, a.value, b.value
+
+    def resume(self, rid, now):
+        return lib().kvr_controller_resume(self._h, rid, now)
+
+    def stats(self):
+        s = ControllerStats()
+        _check(lib().kvr_controller_get_stats(self._h, C.byref(s)))
+        return {n: getattr(s, n) for n, _ in s._fields_ if n != "reserved"}
 
 
 def read_load(device_buf, nbytes, launches, device_sink, stream=None):

@@ -124,3 +124,54 @@ def test_config4_trace_full_geometry():
     print("config 4 trace:", counts, "GB suspended %.1f resumed %.1f" % (sg["bytes_suspended"] / 1e9, sg["bytes_resumed"] / 1e9))
     g.close()
     o.close()
+
+
+def test_live_controller_with_data():
+    """The clock-driven controller (grace period in HBM, offload, one-shot timers, eviction of the longest
+    suspended copy) on the GPU pool, next to the oracle's controller on the CPU pool: same decisions, same cost,
+    and the same bytes in every surviving host image and in the pool at the end."""
+    from kvr_synth import paper_wait_family, poisson_arrivals
+    from oracle.controller import LIVE, TTL, OrcController
+    from test_controller_cpu import PRICES, run_trace
+    geom = (2, 2, 16, 2, 4)                        # 256 bytes per token
+    n, NB, host_cap = 200, 700, 40 * 4096
+    rng = np.random.default_rng(33)
+    lengths = rng.integers(1, 120, size=n)
+    mean_img = float(np.mean(lengths)) * 256
+    w_ref = 1800.0
+    lam = 2.5 * (host_cap / mean_img) / w_ref
+    arrive, wait = poisson_arrivals(n, lam, 33), paper_wait_family("mixture", n, 33)
+    t = Twin(geom, NB, host_cap, seed=33, chunk_bytes=8192, staging_slots=2)
+    L, H, D, e, BS = geom
+    o_view = t.o.data.reshape(2 * L, NB, BS * H * D * e)
+    d_view = t.dev.view(2 * L, NB, BS * H * D * e)
+    fills = {}
+
+    def on_admit(i, blocks):                       # the same fresh bytes on both sides (seeded per admission)
+        k = fills.get(i, 0)
+        fills[i] = k + 1
+        fresh = np.random.default_rng([33, i, k]).integers(0, 256, size=(2 * L, len(blocks), BS * H * D * e), dtype=np.uint8)
+        if pool_is_gpu[0]:
+            d_view[:, torch.from_numpy(blocks.astype(np.int64)).cuda()] = torch.from_numpy(fresh).cuda()
+            torch.cuda.synchronize()
+        else:
+            o_view[:, blocks] = fresh
+    pool_is_gpu = [False]
+    co = OrcController(t.o, PRICES, lam, w_ref, mean_image_bytes=mean_img, hbm_grace_s=20.0, branch=TTL, admission=LIVE)
+    lo = run_trace(co, t.o, arrive, wait, lengths, on_admit=on_admit)
+    pool_is_gpu[0] = True
+    fills.clear()
+    cg = kvr.Controller(t.g, PRICES, lam, w_ref, mean_image_bytes=mean_img, hbm_grace_s=20.0, branch=TTL, admission=kvr.ADMIT_LIVE)
+
+    def on_event(now, kind, i, s):
+        if kind == 1 and s == kvr.OK:
+            assert t.g.wait(i) == kvr.OK
+    lg = run_trace(cg, t.g, arrive, wait, lengths, on_event=on_event, on_admit=on_admit)
+    assert lo == lg
+    so, sg = co.stats(), cg.stats()
+    for k in so:
+        assert sg[k] == pytest.approx(so[k], rel=1e-12), k
+    assert so["resumed_host"] > 20 and so["evicted_lru"] > 0 and so["ttl_expired"] > 0 and so["resumed_hbm"] > 0
+    t.assert_same_pool()
+    cg.close()
+    t.close()

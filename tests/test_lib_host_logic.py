@@ -29,12 +29,13 @@ def test_struct_layouts_match_the_header():
     # sizes the C compiler gives for the header's structs, via a tiny C program
     import subprocess
     import tempfile
-    src = '#include <stdio.h>\n#include "kvr.h"\nint main(){printf("%zu %zu %zu\\n", sizeof(kvr_geometry), sizeof(kvr_config), sizeof(kvr_stats));return 0;}\n'
+    src = '#include <stdio.h>\n#include "kvr.h"\nint main(){printf("%zu %zu %zu %zu %zu %zu\\n", sizeof(kvr_geometry), sizeof(kvr_config), sizeof(kvr_stats), sizeof(kvr_prices), sizeof(kvr_controller_config), sizeof(kvr_controller_stats));return 0;}\n'
     with tempfile.TemporaryDirectory() as d:
         open(os.path.join(d, "t.c"), "w").write(src)
         subprocess.check_call(["gcc", "-std=c11", "-I", os.path.join(ROOT, "include"), "-o", os.path.join(d, "t"), os.path.join(d, "t.c")])
         out = subprocess.check_output([os.path.join(d, "t")]).split()
-    assert [int(x) for x in out] == [C.sizeof(kvr.Geometry), C.sizeof(kvr.Config), C.sizeof(kvr.Stats)]
+    assert [int(x) for x in out] == [C.sizeof(kvr.Geometry), C.sizeof(kvr.Config), C.sizeof(kvr.Stats), C.sizeof(kvr.Prices),
+                                     C.sizeof(kvr.ControllerConfig), C.sizeof(kvr.ControllerStats)]
 
 
 def test_bytes_per_token(golden):
