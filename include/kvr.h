@@ -109,7 +109,7 @@ typedef struct {
   int32_t layout;                    /* KVR_LAYER_MAJOR (0) or KVR_BLOCK_MAJOR */
   void *device_pool;                 /* DEVICE pointer to num_blocks*block_size*bytes_per_token bytes,
                                         256-byte aligned, or NULL: the library allocates and frees it */
-  void *host_arena;                  /* page-locked HOST pointer to host_capacity_bytes bytes, 4096-byte
+  void *host_arena;                  /* page-locked HOST pointer to host_capacity_bytes bytes, 256-byte
                                         aligned, or NULL: the library allocates and frees it */
   const int32_t *initial_free_order; /* permutation of [0, num_blocks) or NULL = 0, 1, 2, ... */
 } kvr_config;

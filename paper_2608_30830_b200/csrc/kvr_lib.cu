@@ -605,8 +605,8 @@ kvr_status create_engine(kvr_pool *p) {
     if (e != cudaSuccess) return fail(KVR_ERR_NOMEM, "cudaHostAlloc(arena, %llu): %s", (unsigned long long)c.host_capacity_bytes, cudaGetErrorString(e));
     p->own_arena = true;
   }
-  if (((uintptr_t)p->d_pool & 255) || ((uintptr_t)p->h_arena & 4095))
-    return fail(KVR_ERR_INVALID_ARG, "device_pool must be 256-byte and host_arena 4096-byte aligned");
+  if (((uintptr_t)p->d_pool & 255) || ((uintptr_t)p->h_arena & 255))
+    return fail(KVR_ERR_INVALID_ARG, "device_pool and host_arena must be 256-byte aligned");
   if (c.route == KVR_ROUTE_MAPPED && p->h_arena) {
     cudaError_t e = cudaHostGetDevicePointer((void **)&p->arena_dev, p->h_arena, 0);
     if (e != cudaSuccess) return fail(KVR_ERR_INVALID_ARG, "host_arena is not mapped page-locked memory: %s", cudaGetErrorString(e));

@@ -162,11 +162,7 @@ def test_live_controller_with_data():
     pool_is_gpu[0] = True
     fills.clear()
     cg = kvr.Controller(t.g, PRICES, lam, w_ref, mean_image_bytes=mean_img, hbm_grace_s=20.0, branch=TTL, admission=kvr.ADMIT_LIVE)
-
-    def on_event(now, kind, i, s):
-        if kind == 1 and s == kvr.OK:
-            assert t.g.wait(i) == kvr.OK
-    lg = run_trace(cg, t.g, arrive, wait, lengths, on_event=on_event, on_admit=on_admit)
+    lg = run_trace(cg, t.g, arrive, wait, lengths, on_admit=on_admit)      # release() waits for a resume in flight
     assert lo == lg
     so, sg = co.stats(), cg.stats()
     for k in so:
