@@ -413,7 +413,7 @@ def run_ours(args):
         if args.kernel == "bulk":
             name = name.replace("move_warp", "move_bulk")
         # DRAM traffic per launch: ncu measured read+write = 0.956 x the algorithmic bytes on a 512 MiB chunk
-        # (profiles/ncu_full_gather_small_case.md); traffic grows in proportion to the bytes of a launch
+        # (ncu --set full capture of the gather on a small case); traffic grows in proportion to the bytes of a launch
         launches = max(d["gather_launches"] if g_gbs <= s_gbs else d["scatter_launches"], 1)
         alg_per_launch = 2 * (d["gather_bytes"] if g_gbs <= s_gbs else d["scatter_bytes"]) / launches
         roofline = {"bound": "hbm", "kernel": name, "achieved": ach, "peak": peak, "unit": "GB/s",

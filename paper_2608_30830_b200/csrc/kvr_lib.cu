@@ -269,7 +269,14 @@ std::vector<uint64_t> chunk_caps(const kvr_pool *p, uint64_t total, bool ramp_up
   std::vector<uint64_t> caps;
   uint64_t sum = 0, c = small;
   while (sum < total) { caps.push_back(c); sum += c; c = c * 2 > big ? big : c * 2; }
-  if (!ramp_up) std::reverse(caps.begin(), caps.end());
+  if (!ramp_up && !caps.empty()) {
+    // mirror image: the ramp must END with the small chunks, so the first chunk takes what the ramp leaves over
+    const uint64_t over = sum - total;
+    uint64_t &largest = caps.back();
+    if (over < largest) largest -= over; else caps.pop_back();
+    std::reverse(caps.begin(), caps.end());
+    if (caps[0] < (uint64_t)p->tile_bytes) caps[0] = align_up(p->tile_bytes, 4096);
+  }
   caps.push_back(small);      // chunks are cut on tile boundaries and may fall a little short: spare room
   return caps;
 }
