@@ -335,8 +335,10 @@ def run_ours(args):
     route = {"staged": kvr.ROUTE_STAGED, "mapped": kvr.ROUTE_MAPPED, "dma2d": kvr.ROUTE_DMA2D}[args.route]
     layout = {"layer": kvr.LAYER_MAJOR, "block": kvr.BLOCK_MAJOR}[args.layout]
     kernel = {"warp": kvr.KERNEL_WARP, "bulk": kvr.KERNEL_BULK}[args.kernel]
+    dev_arena = torch.empty(host_cap, dtype=torch.uint8, device="cuda") if args.arena == "device" else None
     pool = kvr.Pool(*w.geom, w.num_blocks, host_cap, initial_free_order=free_order(seed, w.num_blocks),
                     device=local, device_pool=dev_pool.data_ptr(), route=route, kernel=kernel,
+                    host_arena=dev_arena.data_ptr() if dev_arena is not None else None,
                     chunk_bytes=args.chunk_mib << 20, staging_slots=args.slots, max_ctas=args.max_ctas,
                     flags=kvr.PROFILE, layout=layout)
 
@@ -351,7 +353,7 @@ def run_ours(args):
     occupancy = 1.0 - pool.stats()["blocks_free"] / w.num_blocks
     small = filler_ids[small_k] if small_k is not None else None
 
-    link = link_peak(torch, pool, host_cap) if rank == 0 else None
+    link = link_peak(torch, pool, host_cap) if (rank == 0 and dev_arena is None) else None
 
     def barrier():
         torch.cuda.synchronize()
@@ -466,9 +468,13 @@ def run_ours(args):
 
         sus_gbs = payload_all * K / sus_ms / 1e6
         res_gbs = payload_all * K / res_ms / 1e6
-        host_link = dict(link)
-        host_link.update({"suspend_gbs": sus_gbs, "suspend_frac_of_d2h_peak": sus_gbs / world / link["d2h_best_gbs"],
-                          "resume_gbs": res_gbs, "resume_frac_of_h2d_peak": res_gbs / world / link["h2d_best_gbs"]})
+        if link is None:        # device-memory tier: no host link on the path; the bound is HBM
+            host_link = {"arena": "device memory", "suspend_gbs": sus_gbs, "resume_gbs": res_gbs,
+                         "suspend_frac_of_hbm_peak": 2 * sus_gbs / world / peak, "resume_frac_of_hbm_peak": 2 * res_gbs / world / peak}
+        else:
+            host_link = dict(link)
+            host_link.update({"suspend_gbs": sus_gbs, "suspend_frac_of_d2h_peak": sus_gbs / world / link["d2h_best_gbs"],
+                              "resume_gbs": res_gbs, "resume_frac_of_h2d_peak": res_gbs / world / link["h2d_best_gbs"]})
         cpu = cpu_oracle_sample(w.geom, 256 if args.no_extras else 4096)
         sample = ("one %d-token request of this geometry (%.2f GiB payload): oracle gather then scatter, 1 thread"
                   % (256 if args.no_extras else 4096, cpu["payload_bytes"] / 2**30))
@@ -479,7 +485,7 @@ def run_ours(args):
             "config": {"workload": w.name, "geometry": dict(zip(("layers", "kv_heads", "head_dim", "dtype_bytes", "block_size"), w.geom)),
                        "num_blocks": w.num_blocks, "requests_requested": requested, "requests_run": len(ids),
                        "tokens": int(lens.sum()), "payload_bytes_per_direction": payload,
-                       "occupancy_before_suspend": occupancy, "route": args.route, "layout": args.layout, "kernel": args.kernel,
+                       "occupancy_before_suspend": occupancy, "route": args.route, "arena": args.arena, "layout": args.layout, "kernel": args.kernel,
                        "chunk_mib": args.chunk_mib, "staging_slots": args.slots, "seed": seed,
                        "l2": "inputs (tens of GiB) are far larger than L2; no flush needed",
                        "timing": "value: CUDA events, first enqueued work to last byte landed, summed over the two batched moves of each step; e2e: host clock around the K steps"},
@@ -509,6 +515,8 @@ def main():
     ap.add_argument("--kernel", default="bulk", choices=["warp", "bulk"])
     ap.add_argument("--chunk-mib", type=int, default=512)
     ap.add_argument("--slots", type=int, default=2)
+    ap.add_argument("--arena", default="host", choices=["host", "device"],
+                    help="where the second tier lives: pinned host memory, or device memory (stand-in for a peer GPU)")
     ap.add_argument("--max-ctas", type=int, default=0, help="cap on the movers' grid (0 = fill the GPU)")
     ap.add_argument("--num-blocks", type=int, default=0, help="shrink the pool (profiling captures)")
     ap.add_argument("--requests", type=int, default=0, help="override the request count")

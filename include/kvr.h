@@ -110,7 +110,10 @@ typedef struct {
   void *device_pool;                 /* DEVICE pointer to num_blocks*block_size*bytes_per_token bytes,
                                         256-byte aligned, or NULL: the library allocates and frees it */
   void *host_arena;                  /* page-locked HOST pointer to host_capacity_bytes bytes, 256-byte
-                                        aligned, or NULL: the library allocates and frees it */
+                                        aligned, or NULL: the library allocates and frees it.  A DEVICE
+                                        pointer is accepted too (this GPU's memory, or a peer's with peer
+                                        access enabled): the tier then lives in HBM and images are device
+                                        memory; with KVR_ROUTE_MAPPED the movers write it directly */
   const int32_t *initial_free_order; /* permutation of [0, num_blocks) or NULL = 0, 1, 2, ... */
 } kvr_config;
 

@@ -134,6 +134,7 @@ struct kvr_pool {
   char *d_pool = nullptr; bool own_pool = false;
   char *h_arena = nullptr; bool own_arena = false;
   char *arena_dev = nullptr;              // device alias of the arena (mapped route)
+  bool arena_on_device = false;           // the caller's arena is device memory (local or peer)
   cudaStream_t s_gather = nullptr, s_d2h = nullptr, s_h2d = nullptr, s_scatter = nullptr;
   Ring out_ring, in_ring;
   char *staging = nullptr;
@@ -421,10 +422,10 @@ kvr_status enqueue_dma2d(kvr_pool *p, Op &op, std::vector<Item> &items, bool to_
       char *pool_ptr = p->d_pool + (long long)it.blocks[b] * p->block_stride;
       char *img_ptr = p->h_arena + it.lin_off + (size_t)b * p->BS * p->row;
       if (to_linear) {
-        CU(cudaMemcpy2DAsync(img_ptr, img_pitch, pool_ptr, (size_t)p->plane_stride, width, (size_t)p->planes, cudaMemcpyDeviceToHost, c));
+        CU(cudaMemcpy2DAsync(img_ptr, img_pitch, pool_ptr, (size_t)p->plane_stride, width, (size_t)p->planes, cudaMemcpyDefault, c));
         p->st.d2h_copies++; p->st.d2h_bytes += width * p->planes;
       } else {
-        CU(cudaMemcpy2DAsync(pool_ptr, (size_t)p->plane_stride, img_ptr, img_pitch, width, (size_t)p->planes, cudaMemcpyHostToDevice, c));
+        CU(cudaMemcpy2DAsync(pool_ptr, (size_t)p->plane_stride, img_ptr, img_pitch, width, (size_t)p->planes, cudaMemcpyDefault, c));
         p->st.h2d_copies++; p->st.h2d_bytes += width * p->planes;
       }
     }
@@ -519,7 +520,7 @@ kvr_status enqueue(kvr_pool *p, int kind, std::vector<Item> &items, int route, c
       CU(cudaEventRecord(sl.filled, k));
       CU(cudaStreamWaitEvent(c, sl.filled, 0));
       for (auto &cp : ch.copies) {
-        CU(cudaMemcpyAsync(p->h_arena + cp.lin_off, sl.ptr + cp.slot_off, cp.bytes, cudaMemcpyDeviceToHost, c));
+        CU(cudaMemcpyAsync(p->h_arena + cp.lin_off, sl.ptr + cp.slot_off, cp.bytes, cudaMemcpyDefault, c));
         p->st.d2h_copies++; p->st.d2h_bytes += cp.bytes;
       }
       CU(cudaEventRecord(sl.freed, c));
@@ -527,7 +528,7 @@ kvr_status enqueue(kvr_pool *p, int kind, std::vector<Item> &items, int route, c
     } else {
       if (sl.used) CU(cudaStreamWaitEvent(c, sl.freed, 0));
       for (auto &cp : ch.copies) {
-        CU(cudaMemcpyAsync(sl.ptr + cp.slot_off, p->h_arena + cp.lin_off, cp.bytes, cudaMemcpyHostToDevice, c));
+        CU(cudaMemcpyAsync(sl.ptr + cp.slot_off, p->h_arena + cp.lin_off, cp.bytes, cudaMemcpyDefault, c));
         p->st.h2d_copies++; p->st.h2d_bytes += cp.bytes;
       }
       CU(cudaEventRecord(sl.filled, c));
@@ -614,9 +615,18 @@ kvr_status create_engine(kvr_pool *p) {
   }
   if (((uintptr_t)p->d_pool & 255) || ((uintptr_t)p->h_arena & 255))
     return fail(KVR_ERR_INVALID_ARG, "device_pool and host_arena must be 256-byte aligned");
-  if (c.route == KVR_ROUTE_MAPPED && p->h_arena) {
-    cudaError_t e = cudaHostGetDevicePointer((void **)&p->arena_dev, p->h_arena, 0);
-    if (e != cudaSuccess) return fail(KVR_ERR_INVALID_ARG, "host_arena is not mapped page-locked memory: %s", cudaGetErrorString(e));
+  if (p->h_arena) {
+    // the arena may be pinned host memory (the paper's host tier) or device memory: this GPU's, or a peer's that
+    // this device can address.  Copies use cudaMemcpyDefault, so they follow the pointer wherever it lives.
+    cudaPointerAttributes at{};
+    if (c.host_arena && cudaPointerGetAttributes(&at, p->h_arena) == cudaSuccess && at.type == cudaMemoryTypeDevice) {
+      p->arena_on_device = true;
+      p->arena_dev = p->h_arena;
+    } else if (c.route == KVR_ROUTE_MAPPED) {
+      cudaGetLastError();
+      cudaError_t e = cudaHostGetDevicePointer((void **)&p->arena_dev, p->h_arena, 0);
+      if (e != cudaSuccess) return fail(KVR_ERR_INVALID_ARG, "host_arena is not mapped page-locked memory: %s", cudaGetErrorString(e));
+    }
   }
   int lo = 0, hi = 0;
   CU(cudaDeviceGetStreamPriorityRange(&lo, &hi));

@@ -266,3 +266,29 @@ def test_tiny_config_full_size():
     assert s["bytes_suspended"] == s["bytes_resumed"] == int(lens.sum()) * 32768
     assert s["gather_ms"] > 0 and s["scatter_ms"] > 0
     t.close()
+
+
+@pytest.mark.parametrize("route", [kvr.ROUTE_MAPPED, kvr.ROUTE_STAGED, kvr.ROUTE_DMA2D], ids=["direct", "staged", "strided"])
+def test_arena_in_device_memory(route):
+    """The second tier may be device memory (a stand-in here for a peer GPU's HBM reached over NVLink): same
+    bookkeeping, same image bytes, read back from the device arena."""
+    geom = (4, 2, 64, 2, 16)
+    cap = 1 << 21
+    arena = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+    t = Twin(geom, 96, cap, seed=15, host_arena=arena.data_ptr(), route=route, chunk_bytes=65536)
+    lens = [500, 123, 16, 0, 77]
+    ids = list(range(len(lens)))
+    for rid, n in zip(ids, lens):
+        assert t.both("admit", rid, n)[1][0] == kvr.OK
+    a, b = t.both("suspend_to_host", ids)
+    assert a == b and t.g.wait() == kvr.OK
+    dev_arena = arena.cpu().numpy()
+    for rid in ids:
+        d = t.o.info(rid)[1]
+        off = t.g.info(rid)[1]["arena_offset"]
+        assert off == d["arena_offset"]
+        assert np.array_equal(dev_arena[off:off + d["image_bytes"]], d["image"])
+    a, b = t.both("resume_from_host", ids[::-1])
+    assert a == b
+    t.assert_same_pool()
+    t.close()
