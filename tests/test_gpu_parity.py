@@ -292,3 +292,32 @@ def test_arena_in_device_memory(route):
     assert a == b
     t.assert_same_pool()
     t.close()
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_guard_bands_stay_intact(mode):
+    """Canary regions directly before and after the caller-owned pool and arena must survive a busy script:
+    nothing the movers or the copies do may land outside the two buffers."""
+    geom = SMALL
+    NB, cap, guard = 48, 10 * 4096, 4096
+    bpt = kvr.bytes_per_token(*geom[:4])
+    pool_bytes = NB * geom[4] * bpt
+    dev = torch.full((pool_bytes + 2 * guard,), 0x5A, dtype=torch.uint8, device="cuda")
+    host = torch.full((cap + 2 * guard + 4096,), 0x5A, dtype=torch.uint8).pin_memory()
+    hbase = (host.data_ptr() + guard + 255) // 256 * 256
+    hoff = hbase - host.data_ptr()
+    order = np.random.default_rng(8).permutation(NB).astype(np.int32)
+    g = kvr.Pool(*geom, NB, cap, initial_free_order=order, device_pool=dev.data_ptr() + guard, host_arena=hbase,
+                 chunk_bytes=4096, staging_slots=2, **mode)
+    o = orc.OrcPool(*geom, NB, cap, initial_free_order=order, with_data=False, layout=mode.get("layout", 0))
+    ops = random_script(8, 250, max_tokens=70)
+    la, lb = run_script(o, ops), run_script(g, ops)
+    assert [x[1:3] for x in la] == [x[1:3] for x in lb]
+    assert g.wait() == kvr.OK
+    torch.cuda.synchronize()
+    d = dev.cpu().numpy()
+    assert (d[:guard] == 0x5A).all() and (d[guard + pool_bytes:] == 0x5A).all()
+    h = host.numpy()
+    assert (h[:hoff] == 0x5A).all() and (h[hoff + cap:] == 0x5A).all()
+    assert g.stats()["bytes_suspended"] > 0
+    g.close()
