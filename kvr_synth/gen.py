@@ -41,6 +41,11 @@ CONFIGS = {
                       notes="mixed tiering trace: retain / suspend / expire / resume events"),
     "longctx": Workload("longctx", 32, 8, 128, 2, 8, 147456, 8, ("fixed", 131072),
                         notes="8 x 128k tokens, block_size 8, ids fully shuffled"),
+    # not one of the five benchmark configurations: the paper's own model as one tensor-parallel rank sees it
+    # (Llama-3.1-70B, 80 layers, 8 KV heads / TP4 = 2 per GPU): 512-byte rows, 8 KiB tiles, 80 KiB per token per GPU
+    "paper_70b_tp4": Workload("paper_70b_tp4", 80, 2, 128, 2, 16, 32768, 32,
+                              ("lognormal", 8192, 0.6, 1024, 32768), occupancy=0.70,
+                              notes="per-GPU KV shard of the paper's serving setup; small tiles"),
 }
 
 

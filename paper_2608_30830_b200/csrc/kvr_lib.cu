@@ -443,16 +443,11 @@ kvr_status enqueue_dma2d(kvr_pool *p, Op &op, std::vector<Item> &items, bool to_
 
 // Build and upload the descriptors of a move, then enqueue it.  `to_linear` = gather direction.
 // route: KVR_ROUTE_STAGED, KVR_ROUTE_MAPPED, or 0 for a caller-supplied device buffer (lin_dev).
-kvr_status enqueue(kvr_pool *p, int kind, std::vector<Item> &items, int route, char *lin_dev,
-                   uint64_t block_tag, const std::vector<uint64_t> &arena_waits, Clock::time_point t_call,
-                   uint64_t *out_seq) {
+kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> &items, int route, char *lin_dev,
+                        uint64_t block_tag, const std::vector<uint64_t> &arena_waits, Clock::time_point t_call,
+                        uint64_t *out_seq) {
   const bool to_linear = (kind == OP_SUSPEND || kind == OP_EXPORT);
-  kvr_status s = poll(p);
-  if (s) return s;
-
-  Op op;
-  op.seq = p->next_seq++;
-  op.kind = kind;
+  kvr_status s = KVR_OK;
   if ((s = get_event(p, &op.start)) || (s = get_event(p, &op.read_done)) || (s = get_event(p, &op.done))) return s;
 
   if (route == KVR_ROUTE_DMA2D) return enqueue_dma2d(p, op, items, to_linear, block_tag, arena_waits, t_call, out_seq);
@@ -557,6 +552,26 @@ kvr_status enqueue(kvr_pool *p, int kind, std::vector<Item> &items, int route, c
   return KVR_OK;
 }
 
+// A move that could not be enqueued completely: give back what it took.  The events may already sit in a
+// stream, so they are destroyed (legal while pending) rather than reused.
+void abandon(kvr_pool *p, Op &op) {
+  for (auto &pr : op.prof) { if (pr.first) cudaEventDestroy(pr.first); if (pr.second) cudaEventDestroy(pr.second); }
+  for (auto e : op.chunk_done) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : {op.start, op.read_done, op.done}) if (e) cudaEventDestroy(e);
+  if (op.desc >= 0) p->descs[op.desc].busy = 0;
+}
+
+kvr_status enqueue(kvr_pool *p, int kind, std::vector<Item> &items, int route, char *lin_dev, uint64_t block_tag,
+                   const std::vector<uint64_t> &arena_waits, Clock::time_point t_call, uint64_t *out_seq) {
+  if (kvr_status s = poll(p)) return s;
+  Op op;
+  op.seq = p->next_seq++;
+  op.kind = kind;
+  const kvr_status s = enqueue_impl(p, op, kind, items, route, lin_dev, block_tag, arena_waits, t_call, out_seq);
+  if (s != KVR_OK) abandon(p, op);      // on success the move was handed to p->ops
+  return s;
+}
+
 kvr_status check_pool(kvr_pool *p) { return p ? KVR_OK : fail(KVR_ERR_INVALID_ARG, "pool is NULL"); }
 
 void free_blocks(kvr_pool *p, Request &r, uint64_t tag) {
@@ -649,8 +664,12 @@ kvr_status create_engine(kvr_pool *p) {
   CU(cudaHostAlloc((void **)&p->status_word, 64, cudaHostAllocMapped));
   *p->status_word = 0;
   if (c.kernel == KVR_KERNEL_BULK) {
+    // about 192 KiB of shared memory per SM: 3 stages of up to 32 KiB per pipeline, more pipelines for smaller tiles
+    // (measured on B200: 2 x 3 x 32 KiB for 32 KiB tiles, 8 x 3 x 8 KiB for 8 KiB tiles)
     int piece = p->tile_bytes < 32768 ? p->tile_bytes : 32768;
-    p->bulk = BulkShape{2, 3, piece};
+    int warps = (192 * 1024) / (3 * piece);
+    warps = warps < 2 ? 2 : (warps > 8 ? 8 : warps);
+    p->bulk = BulkShape{warps, 3, piece};
     if (const char *env = getenv("KVR_BULK_SHAPE")) {   // "warps,stages,piece_bytes": tuning knob for benchmarks
       int w, s, b;
       if (sscanf(env, "%d,%d,%d", &w, &s, &b) == 3) p->bulk = BulkShape{w, s, b};
