@@ -321,3 +321,33 @@ def test_guard_bands_stay_intact(mode):
     assert (h[:hoff] == 0x5A).all() and (h[hoff + cap:] == 0x5A).all()
     assert g.stats()["bytes_suspended"] > 0
     g.close()
+
+
+def test_library_owned_pool_and_arena():
+    """device_pool = NULL and host_arena = NULL: the library allocates both.  Content goes in through
+    kvr_import_from_device, so the host image of a request must be exactly the linear bytes that were imported
+    (scatter then gather by the same table is the identity on valid tokens, as the oracle's own round trip shows)."""
+    geom = (4, 8, 128, 2, 16)
+    bpt = kvr.bytes_per_token(*geom[:4])
+    with kvr.Pool(*geom, 300, 64 << 20, initial_free_order=np.random.default_rng(2).permutation(300)) as g:
+        assert g.device_ptr and g.host_arena_ptr
+        lens = [1000, 37, 512]
+        ids = [1, 2, 3]
+        for rid, n in zip(ids, lens):
+            assert g.admit(rid, n)[0] == kvr.OK
+        cap = sum(-(-n * bpt // 256) * 256 for n in lens)
+        src = torch.randint(0, 256, (cap,), dtype=torch.uint8, device="cuda", generator=torch.Generator(device="cuda").manual_seed(4))
+        torch.cuda.synchronize()
+        st, offs = g.import_from_device(ids, src.data_ptr(), cap, kvr.SYNC)
+        assert st == kvr.OK, kvr.last_error()
+        host_src = src.cpu().numpy()
+        assert g.suspend_to_host(ids, kvr.SYNC)[0] == kvr.OK
+        for rid, n, off in zip(ids, lens, offs):
+            assert np.array_equal(g.host_image(rid), host_src[int(off):int(off) + n * bpt])
+        assert g.resume_from_host(ids[::-1], kvr.SYNC)[0] == kvr.OK
+        out = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+        st, offs2 = g.export_to_device(ids, out.data_ptr(), cap, kvr.SYNC)
+        assert st == kvr.OK and offs2.tolist() == offs.tolist()
+        got = out.cpu().numpy()
+        for n, off in zip(lens, offs):
+            assert np.array_equal(got[int(off):int(off) + n * bpt], host_src[int(off):int(off) + n * bpt])
