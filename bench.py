@@ -513,7 +513,7 @@ def main():
     ap.add_argument("--route", default="staged", choices=["staged", "mapped", "dma2d"])
     ap.add_argument("--layout", default="layer", choices=["layer", "block"], help="pool layout: layer-major or block-major")
     ap.add_argument("--kernel", default="bulk", choices=["warp", "bulk"])
-    ap.add_argument("--chunk-mib", type=int, default=512)
+    ap.add_argument("--chunk-mib", type=int, default=1024, help="staging slot size; the library's own default is 512")
     ap.add_argument("--slots", type=int, default=2)
     ap.add_argument("--arena", default="host", choices=["host", "device"],
                     help="where the second tier lives: pinned host memory, or device memory (stand-in for a peer GPU)")

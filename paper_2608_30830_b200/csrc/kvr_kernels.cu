@@ -81,7 +81,9 @@ __device__ __forceinline__ Tile locate(const MoveArgs &a, const long long *cum, 
 // policy: every byte is touched once) before it stores them.
 template <bool GATHER>
 __global__ void __launch_bounds__(kWarpThreads) move_warp_kernel(const MoveArgs a) {
-  __shared__ long long cum[kMaxSegs + 1];
+  // (nsegs + 1) prefix sums, sized at launch: a large static array would shrink the L1 that the loads in flight
+  // (up to 160 KiB per SM) use as landing space
+  extern __shared__ __align__(8) long long cum[];
   scan_segments(a, cum);
   const int lane = threadIdx.x & 31;
   const int warps_per_cta = blockDim.x >> 5;
@@ -278,8 +280,9 @@ cudaError_t launch_move_warp(bool gather, const MoveArgs &a, int grid_limit, int
   const int warps_per_cta = kWarpThreads / 32;
   const long long work_ctas = (a.total_tiles + warps_per_cta - 1) / warps_per_cta;
   const int grid = default_grid(grid_limit, sm_count, ctas_per_sm, work_ctas);
-  if (gather) move_warp_kernel<true><<<grid, kWarpThreads, 0, s>>>(a);
-  else move_warp_kernel<false><<<grid, kWarpThreads, 0, s>>>(a);
+  const size_t smem = sizeof(long long) * (size_t)(a.nsegs + 1);
+  if (gather) move_warp_kernel<true><<<grid, kWarpThreads, smem, s>>>(a);
+  else move_warp_kernel<false><<<grid, kWarpThreads, smem, s>>>(a);
   return cudaGetLastError();
 }
 
