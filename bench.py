@@ -414,15 +414,15 @@ def run_ours(args):
         name, ach = ("kvr::move_warp<gather>", g_gbs) if g_gbs <= s_gbs else ("kvr::move_warp<scatter>", s_gbs)
         if args.kernel == "bulk":
             name = name.replace("move_warp", "move_bulk")
-        # DRAM traffic per launch: ncu measured read+write = 0.956 x the algorithmic bytes on a 512 MiB chunk
+        # DRAM traffic per launch: ncu measured read+write = 0.979 x the algorithmic bytes on a 1 GiB chunk
         # (ncu --set full capture of the gather on a small case); traffic grows in proportion to the bytes of a launch
         launches = max(d["gather_launches"] if g_gbs <= s_gbs else d["scatter_launches"], 1)
         alg_per_launch = 2 * (d["gather_bytes"] if g_gbs <= s_gbs else d["scatter_bytes"]) / launches
         roofline = {"bound": "hbm", "kernel": name, "achieved": ach, "peak": peak, "unit": "GB/s",
                     "frac": ach / peak, "peak_source": peak_kind + " copy bandwidth, read+write bytes",
                     "algorithmic_bytes_per_launch": alg_per_launch,
-                    "traffic": 0.956 * alg_per_launch,
-                    "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum on a 512 MiB chunk, scaled by bytes per launch",
+                    "traffic": 0.979 * alg_per_launch,
+                    "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum on a 1 GiB chunk, scaled by bytes per launch",
                     "gather": {"gbs": g_gbs, "frac": g_gbs / peak, "launches": d["gather_launches"],
                                "avg_us": 1e3 * d["gather_ms"] / max(d["gather_launches"], 1)},
                     "scatter": {"gbs": s_gbs, "frac": s_gbs / peak, "launches": d["scatter_launches"],
