@@ -38,7 +38,8 @@
  *     KVR_SYNC is given.  Bookkeeping (states, block tables, arena offsets) is
  *     final when the call returns; the bytes are final once kvr_wait() on the
  *     request (or KVR_ALL) returns KVR_OK.  Until then kvr_request_info()
- *     reports KVR_SUSPENDING / KVR_RESUMING.  Later calls that touch the same
+ *     reports KVR_SUSPENDING / KVR_RESUMING (unless a later call has already
+ *     changed the settled state, e.g. a resuming request retained again).  Later calls that touch the same
  *     blocks or host bytes are ordered after the move on the device, so the
  *     caller never has to wait for correctness of the library's own moves;
  *   - one caller thread per pool.

@@ -971,7 +971,13 @@ kvr_status kvr_request_info(kvr_pool *p, uint64_t req, int32_t *state, int64_t *
   if (it == p->reqs.end()) return fail(KVR_ERR_UNKNOWN_REQUEST, "unknown request");
   const Request &r = it->second;
   const bool held = r.state == KVR_ACTIVE || r.state == KVR_RETAINED;
-  if (state) *state = (r.pending_op && r.pending_kind) ? r.pending_kind : r.state;
+  if (state) {
+    // a move in flight shows as SUSPENDING / RESUMING until it lands, unless a later call has already moved the
+    // settled state on (a resuming request that was retained again reports RETAINED)
+    const bool transient = r.pending_op && ((r.pending_kind == KVR_SUSPENDING && r.state == KVR_HOST) ||
+                                            (r.pending_kind == KVR_RESUMING && r.state == KVR_ACTIVE));
+    *state = transient ? r.pending_kind : r.state;
+  }
   if (n_tokens) *n_tokens = r.n_tokens;
   if (nb) *nb = r.nb;
   if (blocks && held) {

@@ -351,3 +351,32 @@ def test_library_owned_pool_and_arena():
         got = out.cpu().numpy()
         for n, off in zip(lens, offs):
             assert np.array_equal(got[int(off):int(off) + n * bpt], host_src[int(off):int(off) + n * bpt])
+
+
+@pytest.mark.parametrize("mode", [MODES[1], MODES[3], MODES[6]])
+def test_random_scripts_with_moves_that_stay_in_flight(mode):
+    """The same seeded scripts on images of tens of MiB, so that calls really do arrive while earlier moves are
+    still on the link: bookkeeping as observed (including reported states) and all bytes must still equal the oracle's."""
+    geom = (2, 8, 128, 2, 16)                     # 8 KiB per token, 32 KiB tiles
+    t = Twin(geom, 2048, 300 << 20, seed=2, chunk_bytes=64 << 20, staging_slots=2, **mode)
+    ops = random_script(2002, 160, max_tokens=6000, n_ids=12, batch=4)
+    la, lb = run_script(t.o, ops), run_script(t.g, ops)
+    for (op, sa, pa, snap_a), (_, sb, pb, snap_b) in zip(la, lb):
+        assert (sa, pa) == (sb, pb) and snap_a == snap_b, op
+    t.assert_same_images(range(12))
+    t.assert_same_pool()
+    t.close()
+
+
+def test_retained_while_resuming_reports_retained():
+    geom = (32, 8, 128, 2, 16)
+    bpt = kvr.bytes_per_token(*geom[:4])
+    dev = torch.zeros(1024 * 16 * bpt, dtype=torch.uint8, device="cuda")
+    with kvr.Pool(*geom, 1024, (4096 * bpt) + 4096, device_pool=dev.data_ptr()) as g:
+        assert g.admit(1, 4096)[0] == kvr.OK
+        assert g.suspend_to_host([1], kvr.SYNC)[0] == kvr.OK
+        assert g.resume_from_host([1])[0] == kvr.OK            # ~9 ms on the link
+        assert g.info(1)[1]["state"] in (kvr.RESUMING, kvr.ACTIVE)
+        assert g.retain_in_hbm([1])[0] == kvr.OK               # legal at once: the bookkeeping is settled
+        assert g.info(1)[1]["state"] == kvr.RETAINED
+        assert g.wait(1) == kvr.OK and g.info(1)[1]["state"] == kvr.RETAINED
