@@ -380,3 +380,54 @@ def test_retained_while_resuming_reports_retained():
         assert g.retain_in_hbm([1])[0] == kvr.OK               # legal at once: the bookkeeping is settled
         assert g.info(1)[1]["state"] == kvr.RETAINED
         assert g.wait(1) == kvr.OK and g.info(1)[1]["state"] == kvr.RETAINED
+
+
+def test_admit_waits_for_the_gather_that_still_reads_its_blocks():
+    """A suspend is enqueued and, with no wait, a new request is admitted into exactly the blocks it released and the
+    caller overwrites them at once.  kvr_request_admit must have let the gather finish first: the host image has to
+    hold the old bytes."""
+    geom = (32, 8, 128, 2, 16)
+    bpt = kvr.bytes_per_token(*geom[:4])
+    NB, n = 512, 4096                                       # 256 blocks = 512 MiB per request
+    dev = torch.empty(NB * 16 * bpt, dtype=torch.uint8, device="cuda")
+    dev.view(torch.bfloat16).normal_(generator=torch.Generator(device="cuda").manual_seed(3))
+    tiles = dev.view(2 * 32, NB, 16 * 2048)
+    with kvr.Pool(*geom, NB, n * bpt + 4096, device_pool=dev.data_ptr(), chunk_bytes=32 << 20) as g:
+        a = g.admit(1, n)[1]
+        assert g.admit(2, n)[0] == kvr.OK and g.stats()["blocks_free"] == 0
+        idx = torch.from_numpy(a.astype(np.int64)).cuda()
+        want = tiles.index_select(1, idx).reshape(64, n * 2048).cpu().numpy().reshape(-1)   # the image, by definition
+        torch.cuda.synchronize()
+        assert g.suspend_to_host([1])[0] == kvr.OK           # ~9 ms of link time, gather chunks spread over it
+        st, c = g.admit(3, n)                                # takes the 256 blocks just released
+        assert st == kvr.OK and sorted(c.tolist()) == sorted(a.tolist())
+        tiles[:, idx] = 0xFF                                 # the caller's prefill, on its own stream
+        torch.cuda.synchronize()
+        assert g.wait() == kvr.OK
+        assert np.array_equal(g.host_image(1), want)
+
+
+def test_suspend_into_a_host_range_that_a_resume_is_still_reading():
+    """The arena holds one image.  A resume releases the range at once (bookkeeping) while its copies are still
+    reading it; the next suspend is placed on the same bytes with no wait in between and must not overwrite them early."""
+    geom = (32, 8, 128, 2, 16)
+    bpt = kvr.bytes_per_token(*geom[:4])
+    NB, n = 768, 4096
+    dev = torch.empty(NB * 16 * bpt, dtype=torch.uint8, device="cuda")
+    dev.view(torch.bfloat16).normal_(generator=torch.Generator(device="cuda").manual_seed(5))
+    tiles = dev.view(2 * 32, NB, 16 * 2048)
+
+    def logical(blocks):
+        idx = torch.from_numpy(np.asarray(blocks).astype(np.int64)).cuda()
+        return tiles.index_select(1, idx).reshape(64, n * 2048).cpu().numpy().reshape(-1)
+    for route in (kvr.ROUTE_STAGED, kvr.ROUTE_MAPPED, kvr.ROUTE_DMA2D):
+        with kvr.Pool(*geom, NB, n * bpt, device_pool=dev.data_ptr(), route=route, chunk_bytes=32 << 20) as g:
+            a, b = g.admit(1, n)[1], g.admit(2, n)[1]
+            want_a, want_b = logical(a), logical(b)
+            assert g.suspend_to_host([1], kvr.SYNC)[0] == kvr.OK and g.info(1)[1]["arena_offset"] == 0
+            assert g.suspend_to_host([2])[0] == kvr.HOST_FULL                      # one image fills the tier
+            assert g.resume_from_host([1])[0] == kvr.OK                            # reads [0, 512 MiB) for ~9 ms
+            assert g.suspend_to_host([2])[0] == kvr.OK and g.info(2)[1]["arena_offset"] == 0
+            assert g.wait() == kvr.OK
+            assert np.array_equal(logical(g.info(1)[1]["blocks"]), want_a)         # request 1 came back whole
+            assert np.array_equal(g.host_image(2), want_b)
