@@ -143,6 +143,25 @@ def run_reference(args):
     }))
 
 
+def copy_peak_same_run(torch, nbytes=2 << 30, reps=10):
+    """torch's device-to-device copy on this very GPU, counted read + write like the driver's measured peak."""
+    free_b, _ = torch.cuda.mem_get_info()
+    if free_b < 2 * nbytes + (1 << 30):
+        return None
+    a = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    b = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    ts = []
+    for _ in range(reps + 3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        b.copy_(a)
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    del a, b
+    return 2 * nbytes / min(ts[3:]) / 1e6
+
+
 def link_peak(torch, kvr_pool, arena_bytes, reps=10):
     """Pinned cudaMemcpyAsync peak in each direction over the library's own arena (same placement)."""
     import ctypes as C
@@ -418,7 +437,9 @@ def run_ours(args):
         # (ncu --set full capture of the gather on a small case); traffic grows in proportion to the bytes of a launch
         launches = max(d["gather_launches"] if g_gbs <= s_gbs else d["scatter_launches"], 1)
         alg_per_launch = 2 * (d["gather_bytes"] if g_gbs <= s_gbs else d["scatter_bytes"]) / launches
+        same_run = None if args.no_extras else copy_peak_same_run(torch)
         roofline = {"bound": "hbm", "kernel": name, "achieved": ach, "peak": peak, "unit": "GB/s",
+                    "copy_peak_this_gpu_this_run": same_run,
                     "frac": ach / peak, "peak_source": peak_kind + " copy bandwidth, read+write bytes",
                     "algorithmic_bytes_per_launch": alg_per_launch,
                     "traffic": 0.979 * alg_per_launch,
