@@ -163,32 +163,13 @@ def copy_peak_same_run(torch, nbytes=2 << 30, reps=10):
 
 
 def link_peak(torch, kvr_pool, arena_bytes, reps=10):
-    """Pinned cudaMemcpyAsync peak in each direction over the library's own arena (same placement)."""
-    import ctypes as C
+    """Pinned-copy peak in each direction over the library's own arena (same placement), by the library's probe."""
     n = min(arena_bytes // 4096 * 4096, 2 << 30)
-    host = torch.frombuffer((C.c_uint8 * n).from_address(kvr_pool.host_arena_ptr), dtype=torch.uint8)
-    dev = torch.empty(n, dtype=torch.uint8, device="cuda")
-    out = {"bytes": n, "pinned": bool(host.is_pinned())}
-    s = torch.cuda.Stream()
-    for name in ("d2h", "h2d"):
-        ts = []
-        for _ in range(reps + 3):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            with torch.cuda.stream(s):
-                e0.record()
-                if name == "d2h":
-                    host.copy_(dev, non_blocking=True)
-                else:
-                    dev.copy_(host, non_blocking=True)
-                e1.record()
-            torch.cuda.synchronize()
-            ts.append(e0.elapsed_time(e1))
-        ts = sorted(ts[3:])
-        out[name + "_best_gbs"] = n / ts[0] / 1e6
-        out[name + "_median_gbs"] = n / ts[len(ts) // 2] / 1e6
-    del dev
-    return out
+    st, d2h, h2d = kvr_pool.probe_link(n, reps)
+    if st != 0:
+        raise SystemExit("kvr_probe_link failed with status %d" % st)
+    return {"bytes": n, "reps": reps, "how": "kvr_probe_link: cudaMemcpyAsync arena <-> device, best of reps",
+            "d2h_best_gbs": d2h, "h2d_best_gbs": h2d}
 
 
 def run_longctx(args):
@@ -231,6 +212,7 @@ def run_longctx(args):
                     device_pool=dev_pool.data_ptr(), chunk_bytes=args.chunk_mib << 20, staging_slots=args.slots,
                     kernel={"warp": kvr.KERNEL_WARP, "bulk": kvr.KERNEL_BULK}[args.kernel], max_ctas=args.max_ctas,
                     flags=kvr.PROFILE)
+    link = link_peak(torch, pool, host_cap)            # while the arena is still empty
     ids = list(range(n_req))
     for rid in ids:
         assert pool.admit(rid, n_tok)[0] == kvr.OK
@@ -285,7 +267,6 @@ def run_longctx(args):
     clocks = sampler.stop()
     st = pool.stats()
     peak, peak_kind = peaks()
-    link = link_peak(torch, pool, host_cap)
     out = {
         "metric": "suspend/resume payload GB/s, both directions overlapped beside a synthetic HBM-read load",
         "value": ovl_load["both_directions_gbs"], "unit": "GB/s", "n_gpus": 1, "steps": reps, "warmup": 1,

@@ -279,6 +279,15 @@ kvr_status kvr_wait(kvr_pool *pool, uint64_t req_or_all, int64_t timeout_ms);
  */
 kvr_status kvr_read_load(const void *device_buf, uint64_t bytes, int32_t launches, void *device_sink, void *stream);
 
+/*
+ * The copy benchmark behind the host-resume price beta_2 (Appendix B: one contiguous payload between page-locked
+ * host memory and the device, synchronised before and after, repeated): copies `bytes` (clipped to the arena)
+ * between the pool's own arena and a temporary device buffer, reps times each way after two warm-ups, and reports
+ * the best rate per direction in GB/s (1e9).  This is the link roofline the moves are judged against, measured
+ * on the very memory they use.  The arena must hold no image (KVR_ERR_BAD_STATE otherwise): it is overwritten.
+ */
+kvr_status kvr_probe_link(kvr_pool *pool, uint64_t bytes, int32_t reps, double *d2h_gbs, double *h2d_gbs);
+
 kvr_status kvr_pool_stats(kvr_pool *pool, kvr_stats *out);
 
 /*

@@ -1039,6 +1039,42 @@ int64_t kvr_free_queue(kvr_pool *p, int32_t *out, int64_t cap) {
   return n;
 }
 
+kvr_status kvr_probe_link(kvr_pool *p, uint64_t bytes, int32_t reps, double *d2h_gbs, double *h2d_gbs) {
+  if (kvr_status s = check_pool(p)) return s;
+  if (p->meta_only || !p->h_arena) return fail(KVR_ERR_BAD_STATE, "the pool has no arena to probe");
+  if (reps < 1 || reps > 1000 || bytes < 4096) return fail(KVR_ERR_INVALID_ARG, "reps in [1, 1000], bytes >= 4096");
+  if (kvr_status s = wait_ops(p, 0, 60000)) return s;
+  if (p->arena.used() != 0) return fail(KVR_ERR_BAD_STATE, "the probe overwrites the arena: it must hold no image");
+  if (bytes > p->arena.capacity()) bytes = p->arena.capacity() / 4096 * 4096;
+  char *dev = nullptr;
+  cudaError_t e = cudaMalloc((void **)&dev, bytes);
+  if (e != cudaSuccess) return fail(KVR_ERR_NOMEM, "cudaMalloc(probe, %llu): %s", (unsigned long long)bytes, cudaGetErrorString(e));
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  kvr_status st = KVR_OK;
+  auto run = [&](bool to_host, double *out) -> kvr_status {
+    double best_ms = 1e30;
+    for (int i = 0; i < reps + 2; ++i) {                     // two warm-ups
+      cudaStream_t s = to_host ? p->s_d2h : p->s_h2d;
+      CU(cudaEventRecord(e0, s));
+      if (to_host) CU(cudaMemcpyAsync(p->h_arena, dev, bytes, cudaMemcpyDefault, s));
+      else CU(cudaMemcpyAsync(dev, p->h_arena, bytes, cudaMemcpyDefault, s));
+      CU(cudaEventRecord(e1, s));
+      CU(cudaEventSynchronize(e1));
+      float ms = 0;
+      CU(cudaEventElapsedTime(&ms, e0, e1));
+      if (i >= 2 && ms < best_ms) best_ms = ms;
+    }
+    if (out) *out = (double)bytes / best_ms / 1e6;
+    return KVR_OK;
+  };
+  if ((st = get_event(p, &e0)) == KVR_OK && (st = get_event(p, &e1)) == KVR_OK &&
+      (st = run(true, d2h_gbs)) == KVR_OK)
+    st = run(false, h2d_gbs);
+  put_event(p, e0); put_event(p, e1);
+  cudaFree(dev);
+  return st;
+}
+
 kvr_status kvr_read_load(const void *device_buf, uint64_t bytes, int32_t launches, void *device_sink, void *stream) {
   if (!device_buf || !device_sink || bytes < 16 || launches < 0 || ((uintptr_t)device_buf & 15) || ((uintptr_t)device_sink & 7))
     return fail(KVR_ERR_INVALID_ARG, "kvr_read_load: NULL, misaligned or empty buffer");

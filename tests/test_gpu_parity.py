@@ -431,3 +431,15 @@ def test_suspend_into_a_host_range_that_a_resume_is_still_reading():
             assert g.wait() == kvr.OK
             assert np.array_equal(logical(g.info(1)[1]["blocks"]), want_a)         # request 1 came back whole
             assert np.array_equal(g.host_image(2), want_b)
+
+
+def test_probe_link_measures_the_arena_and_refuses_when_it_holds_images():
+    geom = (4, 8, 128, 2, 16)
+    with kvr.Pool(*geom, 64, 64 << 20) as g:
+        st, d2h, h2d = g.probe_link(32 << 20, 3)
+        assert st == kvr.OK and 1.0 < d2h < 200.0 and 1.0 < h2d < 200.0      # a PCIe link, in GB/s
+        g.admit(1, 100)
+        assert g.suspend_to_host([1], kvr.SYNC)[0] == kvr.OK
+        assert g.probe_link(32 << 20, 3)[0] == kvr.ERR_BAD_STATE
+    with kvr.Pool(*geom, 64, 0) as g:
+        assert g.probe_link()[0] == kvr.ERR_BAD_STATE                         # no arena at all
