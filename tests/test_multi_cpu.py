@@ -59,3 +59,43 @@ def test_two_gloo_ranks_reduce_like_the_benchmark(tmp_path):
                          capture_output=True, text=True, timeout=240)
     assert out.returncode == 0, out.stderr[-2000:]
     assert "RESULT 3000000000.0 2" in out.stdout
+
+
+TP_WORKER = textwrap.dedent("""
+    import hashlib, sys
+    sys.path.insert(0, %r); sys.path.insert(0, %r)
+    import numpy as np
+    from common import random_script, run_script
+    from paper_2608_30830_b200 import kvr
+    from paper_2608_30830_b200.multi import Group
+    g = Group("gloo")
+    # tensor parallel: every rank holds kv_heads / world heads of every token, in its own pool with its own host tier
+    heads = 8 // g.world
+    order = np.random.default_rng(5).permutation(64).astype(np.int32)
+    pool = kvr.Pool(4, heads, 128, 2, 16, 64, 40 * 4096 * heads, initial_free_order=order, flags=kvr.METADATA_ONLY)
+    log = run_script(pool, random_script(5, 300, max_tokens=200))
+    # what must agree across ranks: every status, every block table, the free queue, which requests are where
+    view = [(op, st, per, {k: (v if isinstance(v, int) else (v[0], v[1], v[2], v[5])) for k, v in snap[0].items()}, snap[1])
+            for op, st, per, snap in log]
+    digest = int.from_bytes(hashlib.sha256(repr(view).encode()).digest()[:6], "big")
+    hi, lo = g.max([digest])[0], -g.max([-digest])[0]
+    assert hi == lo == digest, (hi, lo, digest)
+    if g.rank == 0:
+        print("AGREE", g.world, len(log))
+    g.close()
+""")
+
+
+def test_tensor_parallel_ranks_take_identical_decisions(tmp_path):
+    """The bookkeeping is deterministic, so ranks that shard the KV heads and issue the same calls admit, reject and
+    place every request identically without exchanging a byte; the test compares digests over two gloo ranks."""
+    script = tmp_path / "tp_worker.py"
+    script.write_text(TP_WORKER % (ROOT, os.path.join(ROOT, "tests")))
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    out = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+                          "--master-addr", "127.0.0.1", "--master-port", str(port), str(script)],
+                         capture_output=True, text=True, timeout=240)
+    assert out.returncode == 0, out.stderr[-2000:]
+    assert "AGREE 2 300" in out.stdout
