@@ -165,6 +165,9 @@ kvr_status kvr_pool_destroy(kvr_pool *pool);
  * KVR_HBM_FULL, KVR_ERR_BAD_STATE (id exists), KVR_ERR_INVALID_ARG.
  */
 kvr_status kvr_request_admit(kvr_pool *pool, uint64_t req_id, int64_t n_tokens, int32_t *out_blocks, int32_t cap);
+/* Same, into blocks the caller names (an engine with its own allocator mirrors its choice): nb =
+ * ceil(n_tokens/block_size) ids, each currently free, no repeats; the other free ids keep their order. */
+kvr_status kvr_request_admit_into(kvr_pool *pool, uint64_t req_id, int64_t n_tokens, const int32_t *blocks, int32_t nb);
 /* Forget a request in any state; its blocks go to the free tail, its host range is freed. */
 kvr_status kvr_request_release(kvr_pool *pool, uint64_t req_id);
 

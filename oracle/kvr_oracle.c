@@ -274,6 +274,46 @@ int32_t orc_request_admit(orc_pool *p, uint64_t id, int64_t n_tokens, int32_t *o
   return ORC_OK;
 }
 
+/* admission into blocks the caller names (an engine with its own allocator mirrors its choice here):
+ * every block must be free and named once; the other free ids keep their order */
+int32_t orc_request_admit_into(orc_pool *p, uint64_t id, int64_t n_tokens, const int32_t *blocks, int32_t nb) {
+  if (!p || n_tokens < 0 || nb < 0 || (nb > 0 && !blocks)) return ORC_ERR_INVALID_ARG;
+  if ((n_tokens + p->BS - 1) / p->BS != (int64_t)nb) return ORC_ERR_INVALID_ARG;
+  orc_req *r = find_req(p, id);
+  if (r && r->state != ORC_EXPIRED) return ORC_ERR_BAD_STATE;
+  for (int32_t i = 0; i < nb; ++i) {
+    int found = 0;
+    for (int64_t q = 0; q < p->n_free; ++q) if (p->freeq[q] == blocks[i]) found = 1;
+    for (int32_t j = 0; j < i; ++j) if (blocks[j] == blocks[i]) found = 0;
+    if (!found) return ORC_ERR_INVALID_ARG;
+  }
+  if (!r) {
+    if (p->n_reqs == p->cap_reqs) {
+      int64_t nc = p->cap_reqs ? p->cap_reqs * 2 : 16;
+      orc_req *nr = (orc_req *)realloc(p->reqs, sizeof(orc_req) * (size_t)nc);
+      if (!nr) return ORC_ERR_NOMEM;
+      p->reqs = nr; p->cap_reqs = nc;
+    }
+    r = &p->reqs[p->n_reqs++];
+    memset(r, 0, sizeof(*r));
+    r->id = id;
+  }
+  for (int32_t i = 0; i < nb; ++i)
+    for (int64_t q = 0; q < p->n_free; ++q)
+      if (p->freeq[q] == blocks[i]) {
+        memmove(p->freeq + q, p->freeq + q + 1, sizeof(int32_t) * (size_t)(p->n_free - q - 1));
+        p->n_free -= 1;
+        break;
+      }
+  r->state = ORC_ACTIVE;
+  r->n_tokens = n_tokens;
+  r->nb = nb;
+  r->image_bytes = (uint64_t)n_tokens * p->bpt;
+  r->blocks = (int32_t *)malloc(sizeof(int32_t) * (size_t)(nb ? nb : 1));
+  memcpy(r->blocks, blocks, sizeof(int32_t) * (size_t)nb);
+  return ORC_OK;
+}
+
 int32_t orc_request_release(orc_pool *p, uint64_t id) {
   if (!p) return ORC_ERR_INVALID_ARG;
   orc_req *r = find_req(p, id);

@@ -85,6 +85,7 @@ uint8_t *orc_pool_data(orc_pool *);      /* NULL when with_data = 0 */
 uint64_t orc_pool_bytes(orc_pool *);
 
 int32_t orc_request_admit(orc_pool *, uint64_t id, int64_t n_tokens, int32_t *out_blocks, int32_t cap);
+int32_t orc_request_admit_into(orc_pool *, uint64_t id, int64_t n_tokens, const int32_t *blocks, int32_t nb);
 int32_t orc_request_release(orc_pool *, uint64_t id);
 int32_t orc_retain_in_hbm(orc_pool *, const uint64_t *ids, int32_t n, int32_t *per_req);
 int32_t orc_suspend_to_host(orc_pool *, const uint64_t *ids, int32_t n, int32_t *per_req);

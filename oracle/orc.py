@@ -68,6 +68,8 @@ def lib():
         L.orc_pool_bytes.argtypes = [vp]
         L.orc_request_admit.restype = i32
         L.orc_request_admit.argtypes = [vp, u64, i64, pi32, i32]
+        L.orc_request_admit_into.restype = i32
+        L.orc_request_admit_into.argtypes = [vp, u64, i64, pi32, i32]
         L.orc_request_release.restype = i32
         L.orc_request_release.argtypes = [vp, u64]
         for name in ("orc_retain_in_hbm", "orc_suspend_to_host", "orc_expire", "orc_resume_from_host"):
@@ -158,6 +160,10 @@ class OrcPool:
         out = np.zeros(max(nb, 1), dtype=np.int32)
         st = lib().orc_request_admit(self._h, rid, n_tokens, _i32p(out), nb)
         return st, (out[:nb].copy() if st == OK else None)
+
+    def admit_into(self, rid, n_tokens, blocks):
+        blocks = np.ascontiguousarray(blocks, dtype=np.int32)
+        return lib().orc_request_admit_into(self._h, rid, n_tokens, _i32p(blocks), len(blocks))
 
     def release(self, rid):
         return lib().orc_request_release(self._h, rid)

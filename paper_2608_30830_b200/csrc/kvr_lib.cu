@@ -784,6 +784,27 @@ kvr_status kvr_request_admit(kvr_pool *p, uint64_t id, int64_t n_tokens, int32_t
   return KVR_OK;
 }
 
+kvr_status kvr_request_admit_into(kvr_pool *p, uint64_t id, int64_t n_tokens, const int32_t *blocks, int32_t nb) {
+  if (kvr_status s = check_pool(p)) return s;
+  if (n_tokens < 0 || nb < 0 || (nb > 0 && !blocks)) return fail(KVR_ERR_INVALID_ARG, "bad size or block list");
+  if ((n_tokens + p->BS - 1) / p->BS != (int64_t)nb) return fail(KVR_ERR_INVALID_ARG, "nb must equal ceil(n_tokens / block_size)");
+  auto it = p->reqs.find(id);
+  if (it != p->reqs.end() && it->second.state != KVR_EXPIRED) return fail(KVR_ERR_BAD_STATE, "request exists");
+  std::vector<uint8_t> named(p->NB, 0);
+  for (int32_t i = 0; i < nb; ++i) {
+    if (!p->fq.is_free(blocks[i]) || named[blocks[i]]) return fail(KVR_ERR_INVALID_ARG, "block %d is not free or named twice", blocks[i]);
+    named[blocks[i]] = 1;
+  }
+  const uint64_t tag = p->fq.remove(blocks, nb);
+  Request &r = p->reqs[id];
+  r = Request();
+  r.state = KVR_ACTIVE; r.n_tokens = n_tokens; r.nb = nb;
+  r.image_bytes = (uint64_t)n_tokens * p->bpt;
+  r.blocks.assign(blocks, blocks + nb);
+  if (tag && !p->meta_only) return wait_ops(p, tag, 60000, true);     // a gather may still be reading these blocks
+  return KVR_OK;
+}
+
 kvr_status kvr_request_release(kvr_pool *p, uint64_t id) {
   if (kvr_status s = check_pool(p)) return s;
   auto it = p->reqs.find(id);

@@ -69,7 +69,7 @@ class Stats(C.Structure):
 
 
 EXPORTS = [
-    "kvr_bytes_per_token", "kvr_pool_create", "kvr_pool_destroy", "kvr_request_admit", "kvr_request_release",
+    "kvr_bytes_per_token", "kvr_pool_create", "kvr_pool_destroy", "kvr_request_admit", "kvr_request_admit_into", "kvr_request_release",
     "kvr_retain_in_hbm", "kvr_suspend_to_host", "kvr_expire", "kvr_resume_from_host",
     "kvr_resume_from_host_into", "kvr_export_to_device", "kvr_import_from_device", "kvr_request_info",
     "kvr_request_latency", "kvr_wait", "kvr_pool_stats", "kvr_free_queue", "kvr_pool_device_ptr",
@@ -104,6 +104,8 @@ def lib():
     L.kvr_pool_destroy.argtypes = [vp]
     L.kvr_request_admit.restype = i32
     L.kvr_request_admit.argtypes = [vp, u64, i64, pi32, i32]
+    L.kvr_request_admit_into.restype = i32
+    L.kvr_request_admit_into.argtypes = [vp, u64, i64, pi32, i32]
     L.kvr_request_release.restype = i32
     L.kvr_request_release.argtypes = [vp, u64]
     for name in ("kvr_retain_in_hbm", "kvr_expire"):
@@ -339,6 +341,10 @@ class Pool:
         out = np.zeros(max(nb, 1), dtype=np.int32)
         st = lib().kvr_request_admit(self._h, rid, n_tokens, _i32p(out), nb)
         return st, (out[:nb].copy() if st == OK else None)
+
+    def admit_into(self, rid, n_tokens, blocks):
+        blocks = np.ascontiguousarray(blocks, dtype=np.int32)
+        return lib().kvr_request_admit_into(self._h, rid, n_tokens, _i32p(blocks), len(blocks))
 
     def release(self, rid):
         return lib().kvr_request_release(self._h, rid)

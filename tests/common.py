@@ -15,10 +15,12 @@ def random_script(seed, n_ops, max_tokens, n_ids=12, batch=4):
     rng = np.random.default_rng(seed)
     ops = []
     for _ in range(n_ops):
-        kind = rng.choice(["admit", "admit", "retain", "suspend", "suspend", "expire", "resume", "resume",
+        kind = rng.choice(["admit", "admit", "admit_into", "retain", "suspend", "suspend", "expire", "resume", "resume",
                            "resume_into", "release"])
         if kind == "admit":
             ops.append(("admit", int(rng.integers(n_ids)), int(rng.integers(0, max_tokens + 1))))
+        elif kind == "admit_into":
+            ops.append(("admit_into", int(rng.integers(n_ids)), int(rng.integers(0, max_tokens + 1)), int(rng.integers(2**31))))
         elif kind in ("release", "resume_into"):
             ops.append((kind, int(rng.integers(n_ids)), int(rng.integers(2**31))))
         else:
@@ -53,6 +55,14 @@ def run_script(pool, ops, n_ids=12, after_each=None):
         if kind == "admit":
             st, blocks = pool.admit(op[1], op[2])
             per = None if blocks is None else blocks.tolist()
+        elif kind == "admit_into":
+            bs = pool.geom[4]
+            nb = -(-op[2] // bs)
+            fq = pool.free_queue()
+            pick = np.random.default_rng(op[3]).permutation(fq)[:nb]
+            if len(pick) < nb:                       # not enough free blocks: name an invalid list
+                pick = np.concatenate([pick, np.zeros(nb - len(pick), dtype=np.int32) - 1])
+            st = pool.admit_into(op[1], op[2], pick.astype(np.int32))
         elif kind == "release":
             st = pool.release(op[1])
         elif kind == "resume_into":

@@ -77,6 +77,21 @@ def test_resume_into_named_blocks():
     assert p.free_queue().tolist() == [3, 4, 5, 7, 1]       # the others keep their order
 
 
+def test_admit_into_named_blocks():
+    p = mk(NB=8)
+    assert p.admit_into(1, 9, [5, 2]) == orc.ERR_INVALID_ARG            # 9 tokens need 3 blocks
+    assert p.admit_into(1, 9, [5, 2, 2]) == orc.ERR_INVALID_ARG
+    assert p.admit_into(1, 9, [5, 2, 8]) == orc.ERR_INVALID_ARG
+    assert p.admit_into(1, 9, [5, 2, 7]) == orc.OK
+    assert p.info(1)[1]["blocks"].tolist() == [5, 2, 7] and p.free_queue().tolist() == [0, 1, 3, 4, 6]
+    assert p.admit_into(2, 4, [5]) == orc.ERR_INVALID_ARG               # 5 is live now
+    assert p.admit_into(1, 4, [0]) == orc.ERR_BAD_STATE
+    assert p.admit_into(3, 0, []) == orc.OK and p.info(3)[1]["nb"] == 0
+    p.expire([1])
+    assert p.free_queue().tolist() == [0, 1, 3, 4, 6, 5, 2, 7] and p.admit_into(1, 4, [7]) == orc.OK
+    check_invariants(p, [1, 2, 3])
+
+
 # ---- host arena: first fit, 4 KiB granules, worked by hand --------------------------
 
 def test_arena_first_fit_by_hand():
