@@ -42,7 +42,9 @@
  *     changed the settled state, e.g. a resuming request retained again).  Later calls that touch the same
  *     blocks or host bytes are ordered after the move on the device, so the
  *     caller never has to wait for correctness of the library's own moves;
- *   - one caller thread per pool.
+ *   - calls on one pool may come from any thread: they are serialised by a lock inside the pool and make the
+ *     pool's device current for their duration (kvr_wait only takes the lock to look, not while it sleeps).
+ *     kvr_pool_destroy must not race with other calls.  A kvr_controller is single-threaded.
  */
 #ifndef KVR_H
 #define KVR_H

@@ -26,6 +26,7 @@
 #include <cstdio>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <string>
 #include <thread>
 #include <vector>
@@ -145,6 +146,7 @@ struct kvr_pool {
   uint64_t next_seq = 1;
   std::vector<DescBuf> descs;
   std::vector<PendingFree> pending_free;
+  std::mutex mu;                          // every entry point holds it: calls on one pool are serialised
 };
 
 namespace {
@@ -574,6 +576,19 @@ kvr_status enqueue(kvr_pool *p, int kind, std::vector<Item> &items, int route, c
 
 kvr_status check_pool(kvr_pool *p) { return p ? KVR_OK : fail(KVR_ERR_INVALID_ARG, "pool is NULL"); }
 
+// Held for the length of an entry point: serialises callers on the pool and makes the pool's device current
+// on the calling thread (putting the caller's device back on the way out).
+struct Enter {
+  std::unique_lock<std::mutex> lock;
+  int prev = -1;
+  explicit Enter(kvr_pool *p) : lock(p->mu) {
+    if (p->meta_only) return;
+    int cur = -1;
+    if (cudaGetDevice(&cur) == cudaSuccess && cur != p->device && cudaSetDevice(p->device) == cudaSuccess) prev = cur;
+  }
+  ~Enter() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
 void free_blocks(kvr_pool *p, Request &r, uint64_t tag) {
   p->fq.push(r.blocks.data(), r.nb, tag);
   r.blocks.clear(); r.blocks.shrink_to_fit();
@@ -766,6 +781,7 @@ kvr_status kvr_pool_destroy(kvr_pool *p) {
 
 kvr_status kvr_request_admit(kvr_pool *p, uint64_t id, int64_t n_tokens, int32_t *out_blocks, int32_t cap) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   if (n_tokens < 0) return fail(KVR_ERR_INVALID_ARG, "n_tokens < 0");
   const int64_t nb = (n_tokens + p->BS - 1) / p->BS;
   if (out_blocks && cap < nb) return fail(KVR_ERR_INVALID_ARG, "out_blocks too small");
@@ -786,6 +802,7 @@ kvr_status kvr_request_admit(kvr_pool *p, uint64_t id, int64_t n_tokens, int32_t
 
 kvr_status kvr_request_admit_into(kvr_pool *p, uint64_t id, int64_t n_tokens, const int32_t *blocks, int32_t nb) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   if (n_tokens < 0 || nb < 0 || (nb > 0 && !blocks)) return fail(KVR_ERR_INVALID_ARG, "bad size or block list");
   if ((n_tokens + p->BS - 1) / p->BS != (int64_t)nb) return fail(KVR_ERR_INVALID_ARG, "nb must equal ceil(n_tokens / block_size)");
   auto it = p->reqs.find(id);
@@ -807,6 +824,7 @@ kvr_status kvr_request_admit_into(kvr_pool *p, uint64_t id, int64_t n_tokens, co
 
 kvr_status kvr_request_release(kvr_pool *p, uint64_t id) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   auto it = p->reqs.find(id);
   if (it == p->reqs.end()) return fail(KVR_ERR_UNKNOWN_REQUEST, "unknown request");
   Request &r = it->second;
@@ -819,6 +837,7 @@ kvr_status kvr_request_release(kvr_pool *p, uint64_t id) {
 
 kvr_status kvr_retain_in_hbm(kvr_pool *p, const uint64_t *req, int32_t n, kvr_status *per_req) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   if (n < 0 || (n > 0 && !req)) return fail(KVR_ERR_INVALID_ARG, "bad request list");
   Batch b{KVR_OK, per_req};
   for (int32_t i = 0; i < n; ++i) {
@@ -833,6 +852,7 @@ kvr_status kvr_retain_in_hbm(kvr_pool *p, const uint64_t *req, int32_t n, kvr_st
 
 kvr_status kvr_expire(kvr_pool *p, const uint64_t *req, int32_t n, kvr_status *per_req) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   if (n < 0 || (n > 0 && !req)) return fail(KVR_ERR_INVALID_ARG, "bad request list");
   Batch b{KVR_OK, per_req};
   for (int32_t i = 0; i < n; ++i) {
@@ -852,6 +872,7 @@ kvr_status kvr_expire(kvr_pool *p, const uint64_t *req, int32_t n, kvr_status *p
 
 kvr_status kvr_suspend_to_host(kvr_pool *p, const uint64_t *req, int32_t n, uint32_t flags, kvr_status *per_req) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   if (n < 0 || (n > 0 && !req)) return fail(KVR_ERR_INVALID_ARG, "bad request list");
   const auto t_call = Clock::now();
   if (!p->meta_only) { if (kvr_status s = poll(p)) return s; }
@@ -899,6 +920,7 @@ static kvr_status resume_common(kvr_pool *p, std::vector<Item> &items, uint64_t 
 
 kvr_status kvr_resume_from_host(kvr_pool *p, const uint64_t *req, int32_t n, uint32_t flags, kvr_status *per_req) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   if (n < 0 || (n > 0 && !req)) return fail(KVR_ERR_INVALID_ARG, "bad request list");
   const auto t_call = Clock::now();
   Batch b{KVR_OK, per_req};
@@ -927,6 +949,7 @@ kvr_status kvr_resume_from_host(kvr_pool *p, const uint64_t *req, int32_t n, uin
 
 kvr_status kvr_resume_from_host_into(kvr_pool *p, uint64_t req, const int32_t *blocks, int32_t nb, uint32_t flags) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   if (nb < 0 || (nb > 0 && !blocks)) return fail(KVR_ERR_INVALID_ARG, "bad block list");
   const auto t_call = Clock::now();
   auto it = p->reqs.find(req);
@@ -950,6 +973,7 @@ kvr_status kvr_resume_from_host_into(kvr_pool *p, uint64_t req, const int32_t *b
 static kvr_status device_copy(kvr_pool *p, int kind, const uint64_t *req, int32_t n, char *dev, uint64_t capacity,
                               uint64_t *offsets, uint32_t flags) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   if (p->meta_only) return fail(KVR_ERR_BAD_STATE, "metadata-only pool moves no data");
   if (n < 0 || (n > 0 && !req) || !dev || ((uintptr_t)dev & 255)) return fail(KVR_ERR_INVALID_ARG, "bad request list or buffer (256-byte aligned device pointer)");
   const auto t_call = Clock::now();
@@ -987,6 +1011,7 @@ kvr_status kvr_import_from_device(kvr_pool *p, const uint64_t *req, int32_t n, c
 kvr_status kvr_request_info(kvr_pool *p, uint64_t req, int32_t *state, int64_t *n_tokens, int32_t *nb, int32_t *blocks,
                             int32_t cap, const void **host_image, uint64_t *image_bytes, uint64_t *arena_offset) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   if (!p->meta_only) { if (kvr_status s = poll(p)) return s; }
   auto it = p->reqs.find(req);
   if (it == p->reqs.end()) return fail(KVR_ERR_UNKNOWN_REQUEST, "unknown request");
@@ -1013,6 +1038,7 @@ kvr_status kvr_request_info(kvr_pool *p, uint64_t req, int32_t *state, int64_t *
 
 kvr_status kvr_request_latency(kvr_pool *p, uint64_t req, double *host_ms, double *device_ms) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   if (!p->meta_only) { if (kvr_status s = poll(p)) return s; }
   auto it = p->reqs.find(req);
   if (it == p->reqs.end()) return fail(KVR_ERR_UNKNOWN_REQUEST, "unknown request");
@@ -1025,15 +1051,30 @@ kvr_status kvr_request_latency(kvr_pool *p, uint64_t req, double *host_ms, doubl
 kvr_status kvr_wait(kvr_pool *p, uint64_t req_or_all, int64_t timeout_ms) {
   if (kvr_status s = check_pool(p)) return s;
   if (p->meta_only) return KVR_OK;
-  if (req_or_all == KVR_ALL) return wait_ops(p, 0, timeout_ms);
-  auto it = p->reqs.find(req_or_all);
-  if (it == p->reqs.end()) return fail(KVR_ERR_UNKNOWN_REQUEST, "unknown request");
-  if (!it->second.pending_op) return KVR_OK;
-  return wait_ops(p, it->second.pending_op, timeout_ms);
+  if (timeout_ms < 0) timeout_ms = 60000;
+  const auto t0 = Clock::now();
+  // the lock is taken per look, not for the whole wait, so other threads keep working on the pool meanwhile
+  for (unsigned spin = 0;; ++spin) {
+    {
+      Enter enter(p);
+      uint64_t seq = 0;
+      if (req_or_all != KVR_ALL) {
+        auto it = p->reqs.find(req_or_all);
+        if (it == p->reqs.end()) return fail(KVR_ERR_UNKNOWN_REQUEST, "unknown request");
+        seq = it->second.pending_op;
+        if (!seq) return KVR_OK;
+      }
+      const kvr_status s = wait_ops(p, seq, 0);
+      if (s != KVR_ERR_TIMEOUT) return s;
+    }
+    if (ms_since(t0) > (double)timeout_ms) return fail(KVR_ERR_TIMEOUT, "move still in flight after %lld ms", (long long)timeout_ms);
+    if (spin > 2000) std::this_thread::sleep_for(std::chrono::microseconds(50));
+  }
 }
 
 kvr_status kvr_pool_stats(kvr_pool *p, kvr_stats *out) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   if (!out) return fail(KVR_ERR_INVALID_ARG, "out is NULL");
   if (!p->meta_only) { if (kvr_status s = poll(p)) return s; }
   kvr_stats s = p->st;
@@ -1055,6 +1096,7 @@ kvr_status kvr_pool_stats(kvr_pool *p, kvr_stats *out) {
 
 int64_t kvr_free_queue(kvr_pool *p, int32_t *out, int64_t cap) {
   if (!p) return -1;
+  Enter enter(p);
   const int64_t n = p->fq.size();
   if (out) for (int64_t i = 0; i < n && i < cap; ++i) out[i] = p->fq.at(i);
   return n;
@@ -1062,6 +1104,7 @@ int64_t kvr_free_queue(kvr_pool *p, int32_t *out, int64_t cap) {
 
 kvr_status kvr_probe_link(kvr_pool *p, uint64_t bytes, int32_t reps, double *d2h_gbs, double *h2d_gbs) {
   if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
   if (p->meta_only || !p->h_arena) return fail(KVR_ERR_BAD_STATE, "the pool has no arena to probe");
   if (reps < 1 || reps > 1000 || bytes < 4096) return fail(KVR_ERR_INVALID_ARG, "reps in [1, 1000], bytes >= 4096");
   if (kvr_status s = wait_ops(p, 0, 60000)) return s;

@@ -114,3 +114,44 @@ def test_metadata_only_pool_refuses_data_calls():
     st, _ = p.export_to_device([1], 256, 1 << 20)
     assert st == kvr.ERR_BAD_STATE and "metadata-only" in kvr.last_error()
     assert p.wait() == kvr.OK and p.device_ptr is None
+
+
+def test_concurrent_callers_are_serialised():
+    """Four threads work on one pool at once (ctypes drops the GIL during a call), each on its own requests.
+    Every call must see consistent bookkeeping: conservation and disjointness hold at the end and nothing is lost."""
+    import threading
+    NB = 4096
+    p = kvr.Pool(*GEOM, NB, 64 * 4096, flags=kvr.METADATA_ONLY)
+    errors = []
+
+    def worker(base):
+        rng = np.random.default_rng(base)
+        try:
+            for it in range(400):
+                rid = base + int(rng.integers(8))
+                kind = int(rng.integers(6))
+                if kind == 0:
+                    p.admit(rid, int(rng.integers(1, 60)))
+                elif kind == 1:
+                    p.suspend_to_host([rid])
+                elif kind == 2:
+                    p.resume_from_host([rid])
+                elif kind == 3:
+                    p.expire([rid])
+                elif kind == 4:
+                    p.retain_in_hbm([rid])
+                else:
+                    p.release(rid)
+                if it % 50 == 0:
+                    s = p.stats()
+                    assert s["blocks_free"] + s["blocks_active"] + s["blocks_pinned"] == NB
+        except Exception as e:        # surfaced below: an assertion in a thread would otherwise vanish
+            errors.append(e)
+    threads = [threading.Thread(target=worker, args=(100 * k,)) for k in range(1, 5)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    ids = [100 * k + i for k in range(1, 5) for i in range(8)]
+    check_invariants(p, ids)
