@@ -443,3 +443,46 @@ def test_probe_link_measures_the_arena_and_refuses_when_it_holds_images():
         assert g.probe_link(32 << 20, 3)[0] == kvr.ERR_BAD_STATE
     with kvr.Pool(*geom, 64, 0) as g:
         assert g.probe_link()[0] == kvr.ERR_BAD_STATE                         # no arena at all
+
+
+def test_two_threads_move_their_own_requests_concurrently():
+    """Two caller threads suspend and resume disjoint requests on one pool at the same time.  Which blocks and host
+    ranges each move gets depends on the interleaving, so the check is on content: every request comes back whole."""
+    import threading
+    geom = (8, 8, 128, 2, 16)                      # 32 KiB per token
+    bpt = kvr.bytes_per_token(*geom[:4])
+    NB, n = 1024, 1500                             # 94 blocks, 47 MiB per request
+    dev = torch.empty(NB * 16 * bpt, dtype=torch.uint8, device="cuda")
+    dev.view(torch.bfloat16).normal_(generator=torch.Generator(device="cuda").manual_seed(9))
+    tiles = dev.view(2 * 8, NB, 16 * 2048)
+
+    def logical(blocks):
+        idx = torch.from_numpy(np.asarray(blocks).astype(np.int64)).cuda()
+        full = tiles.index_select(1, idx).reshape(16, len(blocks) * 16, 2048)[:, :n]
+        return full.cpu().numpy()
+    with kvr.Pool(*geom, NB, 8 * n * bpt, device_pool=dev.data_ptr(), chunk_bytes=16 << 20,
+                  initial_free_order=np.random.default_rng(9).permutation(NB)) as g:
+        ids = list(range(8))
+        want = {rid: logical(g.admit(rid, n)[1]) for rid in ids}
+        torch.cuda.synchronize()
+        errors = []
+
+        def worker(mine):
+            try:
+                for _ in range(6):
+                    assert g.suspend_to_host(mine)[0] == kvr.OK
+                    assert g.resume_from_host(mine[::-1])[0] == kvr.OK
+                for rid in mine:
+                    assert g.wait(rid, 20000) == kvr.OK
+            except Exception as e:
+                errors.append(e)
+        threads = [threading.Thread(target=worker, args=(ids[:4],)), threading.Thread(target=worker, args=(ids[4:],))]
+        for t in threads:
+            t.start()
+        for t in threads:
+            t.join()
+        assert not errors, errors
+        assert g.wait() == kvr.OK
+        for rid in ids:
+            assert np.array_equal(logical(g.info(rid)[1]["blocks"]), want[rid]), rid
+        check_invariants(g, ids)
