@@ -81,8 +81,7 @@ __device__ __forceinline__ Tile locate(const MoveArgs &a, const long long *cum, 
 // policy: every byte is touched once) before it stores them.
 template <bool GATHER>
 __global__ void __launch_bounds__(kWarpThreads) move_warp_kernel(const MoveArgs a) {
-  // (nsegs + 1) prefix sums, sized at launch: a large static array would shrink the L1 that the loads in flight
-  // (up to 160 KiB per SM) use as landing space
+  // (nsegs + 1) prefix sums, sized at launch (typically a few dozen bytes)
   extern __shared__ __align__(8) long long cum[];
   scan_segments(a, cum);
   const int lane = threadIdx.x & 31;
