@@ -486,3 +486,22 @@ def test_two_threads_move_their_own_requests_concurrently():
         for rid in ids:
             assert np.array_equal(logical(g.info(rid)[1]["blocks"]), want[rid]), rid
         check_invariants(g, ids)
+
+
+@pytest.mark.parametrize("mode", MODES[:4])
+def test_tiles_larger_than_one_bulk_piece(mode):
+    """block_size 64 with 2 KiB rows gives 128 KiB tiles: the bulk mover cuts each into four 32 KiB pieces, and a
+    ragged last block leaves some pieces short or empty."""
+    geom = (2, 8, 128, 2, 64)
+    t = Twin(geom, 64, 8 << 20, seed=17, chunk_bytes=1 << 20, **mode)
+    lens = [100, 64, 1, 65, 17, 0, 127, 640]
+    ids = list(range(len(lens)))
+    for rid, n in zip(ids, lens):
+        assert t.both("admit", rid, n)[1][0] == kvr.OK
+    a, b = t.both("suspend_to_host", ids)
+    assert a == b
+    t.assert_same_images(ids)
+    a, b = t.both("resume_from_host", ids[::-1])
+    assert a == b
+    t.assert_same_pool()
+    t.close()
