@@ -505,3 +505,22 @@ def test_tiles_larger_than_one_bulk_piece(mode):
     assert a == b
     t.assert_same_pool()
     t.close()
+
+
+@pytest.mark.parametrize("geom", [(3, 1, 24, 2, 5), (2, 3, 40, 4, 3), (1, 1, 8, 2, 1)], ids=["row48", "row480-f32", "row16-bs1"])
+@pytest.mark.parametrize("mode", MODES[:3])
+def test_odd_geometries(geom, mode):
+    """Rows that are multiples of 16 bytes but of nothing larger, odd block sizes, 4-byte elements."""
+    t = Twin(geom, 97, 1 << 20, seed=19, chunk_bytes=4096, **mode)
+    rng = np.random.default_rng(19)
+    lens = [int(x) for x in rng.integers(0, 9 * geom[4], size=9)]
+    ids = list(range(len(lens)))
+    for rid, n in zip(ids, lens):
+        assert t.both("admit", rid, n)[1][0] == kvr.OK
+    a, b = t.both("suspend_to_host", ids)
+    assert a == b
+    t.assert_same_images(ids)
+    a, b = t.both("resume_from_host", ids[::-1])
+    assert a == b
+    t.assert_same_pool()
+    t.close()
