@@ -118,6 +118,32 @@ def cpu_oracle_sample(geom, tokens, threads=1):
             "gbs": 2 * payload / (t2 - t0) / 1e9}
 
 
+def cpu_oracle_threads(geom, tokens, threads):
+    """The same oracle loops, one request per thread (the C calls drop the GIL), over one shared host pool."""
+    import oracle as orc
+    L, H, D, e, BS = geom
+    nb = -(-tokens // BS)
+    NB = 2 * nb * threads
+    pool = fill_bytes(SEED, 78, NB * BS * 2 * L * H * D * e, e).copy()
+    perm = np.random.default_rng(SEED + 1).permutation(NB).astype(np.int32)
+    src = [perm[i * nb:(i + 1) * nb] for i in range(threads)]
+    dst = [perm[(threads + i) * nb:(threads + i + 1) * nb] for i in range(threads)]
+
+    def work(i):
+        img = orc.gather(pool, L, H, D, e, BS, NB, src[i], tokens)
+        orc.scatter(pool, img, L, H, D, e, BS, NB, dst[i], tokens)
+    ts = [threading.Thread(target=work, args=(i,)) for i in range(threads)]
+    t0 = time.perf_counter()
+    for t in ts:
+        t.start()
+    for t in ts:
+        t.join()
+    dt = time.perf_counter() - t0
+    payload = threads * tokens * 2 * L * H * D * e
+    return {"value": 2 * payload / dt / 1e9, "unit": "GB/s", "cores": threads, "seconds": dt,
+            "sample": "%d requests of %d tokens, one oracle gather + scatter per thread" % (threads, tokens)}
+
+
 def run_reference(args):
     """Reference arm: the CPU oracle, untuned, on the host cores; every step is a bounded sample."""
     rank = int(os.environ.get("RANK", "0"))
@@ -163,14 +189,22 @@ def copy_peak_same_run(torch, nbytes=2 << 30, reps=10):
     return 2 * nbytes / min(ts[3:]) / 1e6
 
 
-def link_peak(torch, kvr_pool, arena_bytes, reps=10):
-    """Pinned-copy peak in each direction over the library's own arena (same placement), by the library's probe."""
+def link_peak(torch, kvr_pool, arena_bytes, reps=10, payload=0):
+    """Pinned-copy peak in each direction over the library's own arena (same placement), by the library's probe:
+    a 2 GiB copy (the burst figure, the roofline's denominator) and, when a payload size is given, one contiguous
+    copy of that size (what the host side sustains over tens of GiB; on some hosts it is several percent lower)."""
     n = min(arena_bytes // 4096 * 4096, 2 << 30)
     st, d2h, h2d = kvr_pool.probe_link(n, reps)
     if st != 0:
         raise SystemExit("kvr_probe_link failed with status %d" % st)
-    return {"bytes": n, "reps": reps, "how": "kvr_probe_link: cudaMemcpyAsync arena <-> device, best of reps",
-            "d2h_best_gbs": d2h, "h2d_best_gbs": h2d}
+    out = {"bytes": n, "reps": reps, "how": "kvr_probe_link: cudaMemcpyAsync arena <-> device, best of reps",
+           "d2h_best_gbs": d2h, "h2d_best_gbs": h2d}
+    big = min(arena_bytes, payload, 32 << 30) // 4096 * 4096
+    if big > 2 * n:
+        st, d2h_s, h2d_s = kvr_pool.probe_link(big, 2)
+        if st == 0:
+            out.update({"sustained_bytes": big, "d2h_sustained_gbs": d2h_s, "h2d_sustained_gbs": h2d_s})
+    return out
 
 
 def run_longctx(args):
@@ -440,7 +474,7 @@ def run_ours(args):
     occupancy = 1.0 - pool.stats()["blocks_free"] / w.num_blocks
     small = filler_ids[small_k] if small_k is not None else None
 
-    link = link_peak(torch, pool, host_cap) if (rank == 0 and dev_arena is None) else None
+    link = link_peak(torch, pool, host_cap, payload=payload) if (rank == 0 and dev_arena is None) else None
 
     def barrier():
         torch.cuda.synchronize()
@@ -564,6 +598,9 @@ def run_ours(args):
             host_link = dict(link)
             host_link.update({"suspend_gbs": sus_gbs, "suspend_frac_of_d2h_peak": sus_gbs / world / link["d2h_best_gbs"],
                               "resume_gbs": res_gbs, "resume_frac_of_h2d_peak": res_gbs / world / link["h2d_best_gbs"]})
+            if "d2h_sustained_gbs" in link:
+                host_link.update({"suspend_frac_of_d2h_sustained": sus_gbs / world / link["d2h_sustained_gbs"],
+                                  "resume_frac_of_h2d_sustained": res_gbs / world / link["h2d_sustained_gbs"]})
         cpu = cpu_oracle_sample(w.geom, 256 if args.no_extras else 4096)
         sample = ("one %d-token request of this geometry (%.2f GiB payload): oracle gather then scatter, 1 thread"
                   % (256 if args.no_extras else 4096, cpu["payload_bytes"] / 2**30))
@@ -585,7 +622,9 @@ def run_ours(args):
             "clocks": clocks, "roofline": roofline, "kernels_alone": alone, "host_link": host_link,
             "resume_latency_8k": lone,
             "cpu_baseline": {"value": cpu["gbs"], "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample,
-                             "suspend_s": cpu["suspend_s"], "resume_s": cpu["resume_s"]},
+                             "suspend_s": cpu["suspend_s"], "resume_s": cpu["resume_s"],
+                             "all_cores": None if args.no_extras else
+                             cpu_oracle_threads(w.geom, 1024, min(os.cpu_count() or 1, 32))},
         }
         print(json.dumps(out))
     pool.close()
