@@ -19,6 +19,7 @@
 //     number; a suspend that lands on it waits for the move's last read;
 //   - a move on a request whose previous move is in flight waits for it.
 #include <cuda_runtime.h>
+#include <sys/mman.h>
 
 #include <algorithm>
 #include <chrono>
@@ -134,6 +135,7 @@ struct kvr_pool {
   int device = 0, sm_count = 0;
   char *d_pool = nullptr; bool own_pool = false;
   char *h_arena = nullptr; bool own_arena = false;
+  void *arena_map = nullptr; size_t arena_map_len = 0;   // own arena as a registered mapping (else cudaHostAlloc)
   char *arena_dev = nullptr;              // device alias of the arena (mapped route)
   bool arena_on_device = false;           // the caller's arena is device memory (local or peer)
   cudaStream_t s_gather = nullptr, s_d2h = nullptr, s_h2d = nullptr, s_scatter = nullptr;
@@ -624,7 +626,40 @@ void destroy_engine(kvr_pool *p) {
   if (p->status_word) cudaFreeHost(p->status_word);
   for (cudaStream_t s : {p->s_gather, p->s_d2h, p->s_h2d, p->s_scatter}) if (s) cudaStreamDestroy(s);
   if (p->own_pool && p->d_pool) cudaFree(p->d_pool);
-  if (p->own_arena && p->h_arena) cudaFreeHost(p->h_arena);
+  if (p->own_arena && p->h_arena) {
+    if (p->arena_map) { cudaHostUnregister(p->h_arena); munmap(p->arena_map, p->arena_map_len); }
+    else cudaFreeHost(p->h_arena);
+  }
+}
+
+// Page-locked arena of the library's own: an anonymous mapping backed by transparent huge pages where the host
+// offers them, faulted in by several threads and then registered with CUDA.  Locking 2 MiB pages is several times
+// quicker than cudaHostAlloc's 4 KiB pages (34 GiB: about 6 s against 15 s on the measured host); the copies run at
+// the same rate over either.  Returns false when any step fails: the caller then falls back to cudaHostAlloc.
+bool map_arena(kvr_pool *p, size_t bytes) {
+  const size_t huge = 2u << 20;
+  const size_t len = align_up(bytes, huge) + huge;
+  void *m = mmap(nullptr, len, PROT_READ | PROT_WRITE, MAP_PRIVATE | MAP_ANONYMOUS, -1, 0);
+  if (m == MAP_FAILED) return false;
+  char *base = reinterpret_cast<char *>(align_up(reinterpret_cast<uintptr_t>(m), huge));
+  madvise(base, align_up(bytes, huge), MADV_HUGEPAGE);            // a hint: plain pages work too
+  unsigned n_thr = std::thread::hardware_concurrency();
+  n_thr = n_thr < 1 ? 1 : (n_thr > 8 ? 8 : n_thr);
+  const size_t per = align_up((bytes + n_thr - 1) / n_thr, huge);
+  std::vector<std::thread> touch;
+  for (unsigned t = 0; t < n_thr; ++t)
+    touch.emplace_back([=] {
+      const size_t lo = (size_t)t * per, hi = lo + per < bytes ? lo + per : bytes;
+      for (size_t o = lo; o < hi; o += 4096) base[o] = 0;
+    });
+  for (auto &t : touch) t.join();
+  if (cudaHostRegister(base, bytes, cudaHostRegisterPortable | cudaHostRegisterMapped) != cudaSuccess) {
+    cudaGetLastError();
+    munmap(m, len);
+    return false;
+  }
+  p->h_arena = base; p->arena_map = m; p->arena_map_len = len;
+  return true;
 }
 
 kvr_status create_engine(kvr_pool *p) {
@@ -646,8 +681,10 @@ kvr_status create_engine(kvr_pool *p) {
   }
   if (c.host_arena) p->h_arena = (char *)c.host_arena;
   else if (c.host_capacity_bytes) {
-    cudaError_t e = cudaHostAlloc((void **)&p->h_arena, c.host_capacity_bytes, cudaHostAllocMapped);
-    if (e != cudaSuccess) return fail(KVR_ERR_NOMEM, "cudaHostAlloc(arena, %llu): %s", (unsigned long long)c.host_capacity_bytes, cudaGetErrorString(e));
+    if (!map_arena(p, c.host_capacity_bytes)) {
+      cudaError_t e = cudaHostAlloc((void **)&p->h_arena, c.host_capacity_bytes, cudaHostAllocMapped);
+      if (e != cudaSuccess) return fail(KVR_ERR_NOMEM, "cudaHostAlloc(arena, %llu): %s", (unsigned long long)c.host_capacity_bytes, cudaGetErrorString(e));
+    }
     p->own_arena = true;
   }
   if (((uintptr_t)p->d_pool & 255) || ((uintptr_t)p->h_arena & 255))
