@@ -202,8 +202,6 @@ def test_config5_long_context_overlapped_suspend_and_resume():
     free_dev, _ = torch.cuda.mem_get_info()
     while n_req > 2 and (n_req * n_tok * bpt + (24 << 30) > free_dev or n_req * n_tok * bpt + (40 << 30) > host_avail()):
         n_req -= 2
-    # the suite keeps this case to four requests (two out, two in): the full eight is a benchmark run
-    n_req = min(n_req, 4)
     print("longctx: requests_requested=%d requests_run=%d" % (w.n_requests, n_req))
     NB = n_req * (n_tok // w.block_size)
     host_cap = n_req * n_tok * bpt + (64 << 20)
