@@ -480,6 +480,8 @@ def run_ours(args):
         torch.cuda.synchronize()
         group.barrier()
 
+    last_resume_ms = []
+
     def one_step():
         """Returns (device_ms_suspend, device_ms_resume, wall_s)."""
         t0 = time.perf_counter()
@@ -498,7 +500,9 @@ def run_ours(args):
         st, per = pool.resume_from_host(ids)
         assert st == kvr.OK, (st, per, kvr.last_error())
         assert pool.wait() == kvr.OK, kvr.last_error()
-        res = max(pool.latency(r)[2] for r in ids)
+        per_req = [pool.latency(r)[2] for r in ids]
+        last_resume_ms[:] = per_req
+        res = max(per_req)
         return sus, res, time.perf_counter() - t0
 
     for _ in range(args.warmup):
@@ -621,6 +625,12 @@ def run_ours(args):
             "gpu_launches": int(d["gather_launches"] + d["scatter_launches"]),
             "clocks": clocks, "roofline": roofline, "kernels_alone": alone, "host_link": host_link,
             "resume_latency_8k": lone,
+            "resume_latency_in_batch": {
+                "what": "device time from the batched resume's first enqueued work until each request's last byte landed "
+                        "(requests complete in the order given); last timed step",
+                "first_ms": float(min(last_resume_ms)), "median_ms": float(np.median(last_resume_ms)),
+                "last_ms": float(max(last_resume_ms)),
+                "batch_ms_per_8k_tokens": float(max(last_resume_ms)) * 8192.0 / float(lens.sum())},
             "cpu_baseline": {"value": cpu["gbs"], "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample,
                              "suspend_s": cpu["suspend_s"], "resume_s": cpu["resume_s"],
                              "all_cores": None if args.no_extras else
