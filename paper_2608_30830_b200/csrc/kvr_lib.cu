@@ -263,36 +263,41 @@ struct Plan {
   std::vector<int> req_chunk;     // item -> last chunk that holds bytes of it (-1: none)
 };
 
-// Chunk sizes of one staged move.  A suspend starts with a small chunk and doubles up to the slot size,
-// so the first copy over the link starts after a few microseconds of gathering; a resume ends with
-// chunks that halve down to the small size, so little scattering is left after the last copy.  In
-// between, chunks are slot sized: few, large kernel launches.
-std::vector<uint64_t> chunk_caps(const kvr_pool *p, uint64_t total, bool ramp_up) {
+// Chunk sizes of one staged move.  Every move starts with a small chunk and doubles up to the slot size: a
+// suspend's first copy over the link starts after a few microseconds of gathering, and the first requests of a
+// batched resume are complete (and usable) after milliseconds, not after a whole slot.  A resume also ends with
+// chunks that halve down to the small size, so little scattering is left after the last copy.  In between,
+// chunks are slot sized: few, large kernel launches.
+std::vector<uint64_t> chunk_caps(const kvr_pool *p, uint64_t total, bool ramp_down_too) {
   const uint64_t big = p->cfg.chunk_bytes;
   uint64_t small = 32ull << 20;
   if (small < (uint64_t)p->tile_bytes) small = align_up(p->tile_bytes, 4096);
   if (small > big) small = big;
-  std::vector<uint64_t> caps;
-  uint64_t sum = 0, c = small;
-  while (sum < total) { caps.push_back(c); sum += c; c = c * 2 > big ? big : c * 2; }
-  if (!ramp_up && !caps.empty()) {
-    // mirror image: the ramp must END with the small chunks, so the first chunk takes what the ramp leaves over
-    const uint64_t over = sum - total;
-    uint64_t &largest = caps.back();
-    if (over < largest) largest -= over; else caps.pop_back();
-    std::reverse(caps.begin(), caps.end());
-    if (caps[0] < (uint64_t)p->tile_bytes) caps[0] = align_up(p->tile_bytes, 4096);
+  std::vector<uint64_t> front, back;
+  uint64_t used = 0;
+  for (uint64_t c = small; used < total && c < big; c *= 2) {
+    front.push_back(c); used += c;
+    if (ramp_down_too && used < total) { back.push_back(c); used += c; }
   }
+  while (used < total) { front.push_back(big); used += big; }
+  // the largest chunk gives back what the ramps over-provision
+  if (!front.empty()) {
+    const uint64_t over = used - total;
+    uint64_t &largest = front.back();
+    if (over < largest && largest - over >= (uint64_t)p->tile_bytes) largest -= over;
+  }
+  std::vector<uint64_t> caps(front);
+  caps.insert(caps.end(), back.rbegin(), back.rend());
   caps.push_back(small);      // chunks are cut on tile boundaries and may fall a little short: spare room
   return caps;
 }
 
 // Staged route: cut the concatenated images into chunks on tile boundaries; chunk k goes to slot
 // (ring.next + k) mod slots and holds at most caps[k] bytes.
-void plan_staged(kvr_pool *p, const std::vector<Item> &items, Ring &ring, bool ramp_up, const char *desc_dev, Plan &pl) {
+void plan_staged(kvr_pool *p, const std::vector<Item> &items, Ring &ring, bool ramp_down_too, const char *desc_dev, Plan &pl) {
   uint64_t total = 0;
   for (auto &it : items) total += (uint64_t)it.n_tokens * p->bpt;
-  const std::vector<uint64_t> caps = chunk_caps(p, total, ramp_up);
+  const std::vector<uint64_t> caps = chunk_caps(p, total, ramp_down_too);
   const int nslots = (int)ring.slots.size();
   Chunk cur;
   uint64_t fill = 0, cap = caps[0];
@@ -465,7 +470,7 @@ kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> &items,
   Ring *ring = nullptr;
   if (route == KVR_ROUTE_STAGED) {
     ring = to_linear ? &p->out_ring : &p->in_ring;
-    plan_staged(p, items, *ring, to_linear, nullptr, pl);
+    plan_staged(p, items, *ring, !to_linear, nullptr, pl);
   } else {
     plan_direct(p, items, route == KVR_ROUTE_MAPPED ? p->arena_dev : lin_dev, nullptr, pl);
   }
