@@ -116,7 +116,30 @@ class Rig:
         cleanup()
 
 
-def suspend_resume_checked(rig, ids, whole=None, k=1536):
+def untouched_rows(rig, ids, others, k=256):
+    """Oracle-addressed rows a resume of `ids` must leave alone (same tuple shape as Rig.sample: offset at [4])."""
+    L, H, D, e, BS = rig.geom
+    out = []
+    for rid in ids:                                   # tail slots of a partial last block
+        d = rig.o.info(rid)[1]
+        n = d["n_tokens"]
+        if n % BS:
+            l, kv = int(rig.rng.integers(L)), int(rig.rng.integers(2))
+            for slot in {n % BS, BS - 1}:
+                out.append((rid, l, kv, -1, orc.pool_offset(L, H, D, e, BS, rig.NB, l, kv, int(d["blocks"][-1]), slot), 0))
+    pool_blocks = list(rig.o.free_queue()[:64])       # blocks still free after the resume
+    for rid in others[:8]:                            # blocks of other live requests
+        pool_blocks += list(rig.o.info(rid)[1]["blocks"][:8])
+    for _ in range(k):
+        if not pool_blocks:
+            break
+        blk = int(rig.rng.choice(pool_blocks))
+        l, kv, slot = int(rig.rng.integers(L)), int(rig.rng.integers(2)), int(rig.rng.integers(BS))
+        out.append((-1, l, kv, -1, orc.pool_offset(L, H, D, e, BS, rig.NB, l, kv, blk, slot), 0))
+    return out
+
+
+def suspend_resume_checked(rig, ids, whole=None, k=1536, others=()):
     samples = rig.sample(ids, k)
     before = rig.read_pool_rows(samples)
     want_whole = rig.whole_request_image(whole) if whole is not None else None
@@ -129,9 +152,16 @@ def suspend_resume_checked(rig, ids, whole=None, k=1536):
         assert np.array_equal(rig.g.host_image(whole), want_whole)
     for rid in ids:
         assert rig.o.info(rid)[1]["arena_offset"] == rig.g.info(rid)[1]["arena_offset"]
-    st, per = rig.both("resume_from_host", ids)
-    assert st == kvr.OK
+    # the oracle resumes first: its new tables name the rows that must NOT change -- the slots behind the last valid
+    # token of a partial last block, and rows of blocks that stay free or belong to other requests
+    ro = rig.o.resume_from_host(ids)
+    untouched = untouched_rows(rig, ids, others)
+    keep = rig.read_pool_rows(untouched) if untouched else None
+    rg = rig.g.resume_from_host(ids)
+    assert ro == rg and rg[0] == kvr.OK
     assert rig.g.wait() == kvr.OK, kvr.last_error()
+    if untouched:
+        assert np.array_equal(rig.read_pool_rows(untouched), keep)
     for rid in ids:
         assert rig.o.info(rid)[1]["blocks"].tolist() == rig.g.info(rid)[1]["blocks"].tolist()
     after = rig.resample_pool_offsets(samples)
@@ -158,7 +188,7 @@ def test_config2_llama3_8b_shaped_full_size():
     for rid, n in order:
         assert rig.both("admit", rid, n)[0] == kvr.OK
     assert abs(1 - rig.g.stats()["blocks_free"] / w.num_blocks - 0.70) < 0.001
-    suspend_resume_checked(rig, ids, whole=int(np.argmin(lens)))
+    suspend_resume_checked(rig, ids, whole=int(np.argmin(lens)), others=[1000 + i for i in range(len(fillers))])
     s = rig.g.stats()
     assert s["bytes_suspended"] == s["bytes_resumed"] == s["gather_bytes"] == s["scatter_bytes"] == int(lens.sum()) * bpt
     check_invariants(rig.g, ids + [1000 + i for i in range(len(fillers))])
@@ -187,7 +217,7 @@ def test_config3_gqa64_resume_burst():
         if rig.o.stats()["blocks_free"] > (n_req - rid) * 1024 + 600:
             assert rig.both("admit", fid, 4096)[0] == kvr.OK
             fid += 1
-    suspend_resume_checked(rig, ids, whole=None, k=1024)
+    suspend_resume_checked(rig, ids, whole=None, k=1024, others=list(range(1000, fid)))
     rig.close()
 
 
