@@ -701,6 +701,17 @@ kvr_status create_engine(kvr_pool *p) {
     if (c.host_arena && cudaPointerGetAttributes(&at, p->h_arena) == cudaSuccess && at.type == cudaMemoryTypeDevice) {
       p->arena_on_device = true;
       p->arena_dev = p->h_arena;
+      if (at.device != c.device) {
+        // a peer's memory: make it addressable from this device (plain loads, stores and copies only -- the movers
+        // use no multicast).  "Already enabled" is fine.
+        cudaError_t pe = cudaDeviceEnablePeerAccess(at.device, 0);
+        if (pe != cudaSuccess && pe != cudaErrorPeerAccessAlreadyEnabled) {
+          cudaGetLastError();
+          return fail(KVR_ERR_INVALID_ARG, "host_arena lives on device %d, which device %d cannot address: %s",
+                      at.device, c.device, cudaGetErrorString(pe));
+        }
+        cudaGetLastError();
+      }
     } else if (c.route == KVR_ROUTE_MAPPED) {
       cudaGetLastError();
       cudaError_t e = cudaHostGetDevicePointer((void **)&p->arena_dev, p->h_arena, 0);
