@@ -155,3 +155,46 @@ def test_concurrent_callers_are_serialised():
     assert not errors, errors
     ids = [100 * k + i for k in range(1, 5) for i in range(8)]
     check_invariants(p, ids)
+
+
+def test_a_plain_c_program_can_drive_the_library(tmp_path):
+    """The boundary is a C ABI: compile a C11 program against include/kvr.h, link libkvr.so, run a bookkeeping flow."""
+    import subprocess
+    src = r'''
+    #include <stdio.h>
+    #include <math.h>
+    #include "kvr.h"
+    int main(void) {
+      kvr_config cfg = {0};
+      cfg.g = (kvr_geometry){ .layers = 2, .kv_heads = 2, .head_dim = 4, .dtype_bytes = 2, .block_size = 4 };
+      cfg.num_blocks = 8; cfg.host_capacity_bytes = 1 << 16; cfg.flags = KVR_METADATA_ONLY;
+      kvr_pool *pool = NULL;
+      if (kvr_pool_create(&cfg, &pool) != KVR_OK) { printf("create: %s\n", kvr_last_error()); return 1; }
+      int32_t blocks[3] = {5, 2, 7}, got[3];
+      uint64_t req = 42;
+      if (kvr_request_admit_into(pool, req, 9, blocks, 3) != KVR_OK) return 2;
+      if (kvr_suspend_to_host(pool, &req, 1, KVR_SYNC, NULL) != KVR_OK) return 3;
+      if (kvr_expire(pool, &req, 1, NULL) != KVR_OK) return 4;
+      if (kvr_resume_from_host(pool, &req, 1, 0, NULL) != KVR_RECOMPUTE) return 5;
+      if (kvr_request_admit(pool, req, 9, got, 3) != KVR_OK) return 6;
+      kvr_stats st;
+      kvr_pool_stats(pool, &st);
+      kvr_prices pr = {0.0176, 0.02, 1.91};
+      double t1, ts, t2;
+      kvr_policy_break_evens(&pr, &t1, &ts);
+      kvr_policy_host_ttl(&pr, 2 * 425.0 / 1800.0, 425.0, 1800.0, NULL, &t2);
+      printf("%lld %lld %d %d %d %.3f %.1f %.1f %llu\n", (long long)st.blocks_free, (long long)st.recompute_marked,
+             got[0], got[1], got[2], t1, ts, t2, (unsigned long long)kvr_bytes_per_token(&cfg.g));
+      return kvr_pool_destroy(pool);
+    }
+    '''
+    c = tmp_path / "t.c"
+    c.write_text(src)
+    exe = tmp_path / "t"
+    pkg = os.path.join(ROOT, "paper_2608_30830_b200")
+    kvr.lib()
+    subprocess.check_call(["gcc", "-std=c11", "-I", os.path.join(ROOT, "include"), str(c), "-o", str(exe),
+                           "-L", pkg, "-l:libkvr.so", "-Wl,-rpath," + pkg, "-lm"])
+    out = subprocess.check_output([str(exe)], text=True).split()
+    # free queue after the flow: 0 1 3 4 6 5 2 7 -> admit takes 0 1 3; five blocks stay free
+    assert out == ["5", "1", "0", "1", "3", "1.136", "108.5", "1781.2", "64"]
