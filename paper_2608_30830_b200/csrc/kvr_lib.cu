@@ -642,6 +642,15 @@ void destroy_engine(kvr_pool *p) {
 // quicker than cudaHostAlloc's 4 KiB pages (34 GiB: about 6 s against 15 s on the measured host); the copies run at
 // the same rate over either.  Returns false when any step fails: the caller then falls back to cudaHostAlloc.
 bool map_arena(kvr_pool *p, size_t bytes) {
+  // touching more memory than the host can give would invite the OOM killer; cudaHostAlloc fails politely instead
+  unsigned long long avail_kb = 0;
+  if (FILE *f = fopen("/proc/meminfo", "r")) {
+    char line[256];
+    while (fgets(line, sizeof line, f))
+      if (sscanf(line, "MemAvailable: %llu kB", &avail_kb) == 1) break;
+    fclose(f);
+  }
+  if (!avail_kb || (double)bytes > 0.9 * 1024.0 * (double)avail_kb) return false;
   const size_t huge = 2u << 20;
   const size_t len = align_up(bytes, huge) + huge;
   void *m = mmap(nullptr, len, PROT_READ | PROT_WRITE, MAP_PRIVATE | MAP_ANONYMOUS, -1, 0);

@@ -524,3 +524,10 @@ def test_odd_geometries(geom, mode):
     assert a == b
     t.assert_same_pool()
     t.close()
+
+
+def test_an_arena_larger_than_host_memory_is_refused_politely():
+    avail = int(open("/proc/meminfo").read().split("MemAvailable:")[1].split()[0]) * 1024
+    with pytest.raises(kvr.KvrError) as e:
+        kvr.Pool(4, 8, 128, 2, 16, 64, 4 * avail)
+    assert e.value.status == kvr.ERR_NOMEM
