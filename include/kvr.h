@@ -293,6 +293,16 @@ kvr_status kvr_read_load(const void *device_buf, uint64_t bytes, int32_t launche
  */
 kvr_status kvr_probe_link(kvr_pool *pool, uint64_t bytes, int32_t reps, double *d2h_gbs, double *h2d_gbs);
 
+/*
+ * Self-test of the movers' give-up path (no counterpart in the paper).  Every wait inside the bulk mover is bounded;
+ * when one runs out the kernel writes the pool's device-error word and returns, and kvr_wait() then reports
+ * KVR_ERR_CUDA.  This call makes a wait run out on purpose and safely: one thread polls, 4096 times, a barrier that
+ * nothing completes.  KVR_OK means the thread gave up and the word was written.  With leave_error_set != 0 the word
+ * stays set so that the reporting through kvr_wait() can be observed; kvr_clear_device_error() resets it.
+ */
+kvr_status kvr_selftest_bounded_wait(kvr_pool *pool, int32_t leave_error_set);
+kvr_status kvr_clear_device_error(kvr_pool *pool);
+
 kvr_status kvr_pool_stats(kvr_pool *pool, kvr_stats *out);
 
 /*

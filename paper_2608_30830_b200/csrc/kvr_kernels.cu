@@ -124,8 +124,8 @@ __device__ __forceinline__ bool mbar_test(unsigned bar, unsigned parity) {
   return ok != 0;
 }
 // Bounded wait: false when the limit ran out (the caller records it and leaves).
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
-  for (unsigned spin = 0; spin < kSpinLimit; ++spin) {
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, unsigned limit = kSpinLimit) {
+  for (unsigned spin = 0; spin < limit; ++spin) {
     if (mbar_test(bar, parity)) return true;
     if (spin > 64) __nanosleep(32);
   }
@@ -239,6 +239,20 @@ __global__ void __launch_bounds__(256) read_load_kernel(const uint4 *buf, unsign
   if ((threadIdx.x & 31) == 0) atomicXor(sink + (blockIdx.x & 1023), (unsigned long long)acc);
 }
 
+// Self-test of the give-up path: one thread waits, with a small limit, on an mbarrier that nothing will ever
+// complete; the wait must run out, the thread records it in the status word and returns.
+__global__ void wait_limit_probe_kernel(int *status, unsigned limit) {
+  __shared__ __align__(8) unsigned long long bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_addr(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait(smem_addr(&bar), 0, limit)) {
+      *reinterpret_cast<volatile int *>(status) = 2;
+      __threadfence_system();
+    }
+  }
+}
+
 int default_grid(int grid_limit, int sm_count, int ctas_per_sm, long long work_ctas) {
   long long g = (long long)sm_count * ctas_per_sm;
   if (grid_limit > 0 && g > grid_limit) g = grid_limit;
@@ -291,6 +305,11 @@ cudaError_t launch_read_load(const void *buf, unsigned long long bytes, int laun
   if (ctas < 1 || ctas > 0x7fffffffull) return cudaErrorInvalidValue;
   for (int i = 0; i < launches; ++i)
     read_load_kernel<<<(unsigned)ctas, 256, 0, s>>>(static_cast<const uint4 *>(buf), nvec, static_cast<unsigned long long *>(sink));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_wait_limit_probe(int *status, unsigned limit, cudaStream_t s) {
+  wait_limit_probe_kernel<<<1, 32, 0, s>>>(status, limit);
   return cudaGetLastError();
 }
 

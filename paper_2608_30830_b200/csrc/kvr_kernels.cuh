@@ -50,4 +50,7 @@ cudaError_t bulk_configure(const BulkShape &shape);   // once per device: opt in
 // `launches` back-to-back streaming reads of buf (benchmark load); sink = 8 KiB of device memory
 cudaError_t launch_read_load(const void *buf, unsigned long long bytes, int launches, void *sink, cudaStream_t s);
 
+// one thread waits `limit` polls on an mbarrier nobody completes, then writes 2 to *status (pinned host word)
+cudaError_t launch_wait_limit_probe(int *status, unsigned limit, cudaStream_t s);
+
 }  // namespace kvr

@@ -1175,6 +1175,27 @@ int64_t kvr_free_queue(kvr_pool *p, int32_t *out, int64_t cap) {
   return n;
 }
 
+kvr_status kvr_selftest_bounded_wait(kvr_pool *p, int32_t leave_error_set) {
+  if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
+  if (p->meta_only) return fail(KVR_ERR_BAD_STATE, "metadata-only pool has no device side");
+  if (kvr_status s = wait_ops(p, 0, 60000)) return s;
+  cudaError_t e = launch_wait_limit_probe(p->status_word, 4096, p->s_gather);
+  if (e != cudaSuccess) return fail(KVR_ERR_CUDA, "probe launch: %s", cudaGetErrorString(e));
+  CU(cudaStreamSynchronize(p->s_gather));
+  const int seen = *(volatile int *)p->status_word;
+  if (!leave_error_set) *p->status_word = 0;
+  if (seen != 2) return fail(KVR_ERR_CUDA, "the bounded wait did not run out (status word %d)", seen);
+  return KVR_OK;
+}
+
+kvr_status kvr_clear_device_error(kvr_pool *p) {
+  if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
+  if (p->status_word) *p->status_word = 0;
+  return KVR_OK;
+}
+
 kvr_status kvr_probe_link(kvr_pool *p, uint64_t bytes, int32_t reps, double *d2h_gbs, double *h2d_gbs) {
   if (kvr_status s = check_pool(p)) return s;
   Enter enter(p);

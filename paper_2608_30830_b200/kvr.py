@@ -73,7 +73,7 @@ EXPORTS = [
     "kvr_retain_in_hbm", "kvr_suspend_to_host", "kvr_expire", "kvr_resume_from_host",
     "kvr_resume_from_host_into", "kvr_export_to_device", "kvr_import_from_device", "kvr_request_info",
     "kvr_request_latency", "kvr_wait", "kvr_pool_stats", "kvr_free_queue", "kvr_pool_device_ptr",
-    "kvr_pool_host_arena", "kvr_last_error", "kvr_gather_noalloc", "kvr_read_load", "kvr_probe_link",
+    "kvr_pool_host_arena", "kvr_last_error", "kvr_gather_noalloc", "kvr_read_load", "kvr_probe_link", "kvr_selftest_bounded_wait", "kvr_clear_device_error",
     "kvr_policy_break_evens", "kvr_policy_host_ttl", "kvr_policy_replay", "kvr_policy_select",
     "kvr_controller_create", "kvr_controller_destroy", "kvr_controller_calibrate", "kvr_controller_suspend",
     "kvr_controller_advance", "kvr_controller_resume", "kvr_controller_get_stats",
@@ -161,6 +161,10 @@ def lib():
     L.kvr_controller_resume.argtypes = [vp, u64, C.c_double]
     L.kvr_controller_get_stats.restype = i32
     L.kvr_controller_get_stats.argtypes = [vp, C.POINTER(ControllerStats)]
+    L.kvr_selftest_bounded_wait.restype = i32
+    L.kvr_selftest_bounded_wait.argtypes = [vp, i32]
+    L.kvr_clear_device_error.restype = i32
+    L.kvr_clear_device_error.argtypes = [vp]
     L.kvr_probe_link.restype = i32
     L.kvr_probe_link.argtypes = [vp, u64, i32, pd, pd]
     L.kvr_read_load.restype = i32
@@ -425,6 +429,12 @@ class Pool:
         if st != OK:
             raise KvrError(st, last_error())
         return s.as_dict()
+
+    def selftest_bounded_wait(self, leave_error_set=False):
+        return lib().kvr_selftest_bounded_wait(self._h, int(leave_error_set))
+
+    def clear_device_error(self):
+        return lib().kvr_clear_device_error(self._h)
 
     def probe_link(self, nbytes=2 << 30, reps=10):
         """kvr_probe_link: best pinned-copy rate per direction over this pool's arena, GB/s."""

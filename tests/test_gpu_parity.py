@@ -531,3 +531,22 @@ def test_an_arena_larger_than_host_memory_is_refused_politely():
     with pytest.raises(kvr.KvrError) as e:
         kvr.Pool(4, 8, 128, 2, 16, 64, 4 * avail)
     assert e.value.status == kvr.ERR_NOMEM
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_pool_stays_usable():
+    """The give-up path of the movers, made to happen safely: a thread polls a barrier nothing completes, gives up
+    after its limit, writes the error word; kvr_wait reports it; after clearing, moves work as before."""
+    geom = (4, 2, 64, 2, 16)
+    t = Twin(geom, 64, 1 << 21, seed=23)
+    assert t.g.selftest_bounded_wait() == kvr.OK and t.g.wait() == kvr.OK            # word cleared by the self-test
+    assert t.g.selftest_bounded_wait(leave_error_set=True) == kvr.OK
+    assert t.g.wait() == kvr.ERR_CUDA and "bounded wait" in kvr.last_error()
+    assert t.g.clear_device_error() == kvr.OK and t.g.wait() == kvr.OK
+    t.both("admit", 1, 300)
+    a, b = t.both("suspend_to_host", [1])
+    assert a == b
+    t.assert_same_images([1])
+    a, b = t.both("resume_from_host", [1])
+    assert a == b
+    t.assert_same_pool()
+    t.close()
