@@ -497,7 +497,7 @@ def run_ours(args):
             assert pool.expire([small])[0] == kvr.OK
             assert pool.resume_from_host([small])[0] == kvr.RECOMPUTE
             assert pool.admit(small, small_tokens)[0] == kvr.OK
-        st, per = pool.resume_from_host(ids)
+        st, per = pool.resume_from_host(ids, kvr.LOW_LATENCY if args.low_latency else 0)
         assert st == kvr.OK, (st, per, kvr.last_error())
         assert pool.wait() == kvr.OK, kvr.last_error()
         per_req = [pool.latency(r)[2] for r in ids]
@@ -616,7 +616,7 @@ def run_ours(args):
                        "num_blocks": w.num_blocks, "requests_requested": requested, "requests_run": len(ids),
                        "tokens": int(lens.sum()), "payload_bytes_per_direction": payload,
                        "occupancy_before_suspend": occupancy, "route": args.route, "arena": args.arena, "layout": args.layout, "kernel": args.kernel,
-                       "chunk_mib": args.chunk_mib, "staging_slots": args.slots, "seed": seed,
+                       "chunk_mib": args.chunk_mib, "staging_slots": args.slots, "low_latency_resume": bool(args.low_latency), "seed": seed,
                        "l2": "inputs (tens of GiB) are far larger than L2; no flush needed",
                        "timing": "value: CUDA events, first enqueued work to last byte landed, summed over the two batched moves of each step; e2e: host clock around the K steps"},
             "e2e": {"value": e2e, "unit": "GB/s",
@@ -659,6 +659,7 @@ def main():
     ap.add_argument("--num-blocks", type=int, default=0, help="shrink the pool (profiling captures)")
     ap.add_argument("--requests", type=int, default=0, help="override the request count")
     ap.add_argument("--fixed-tokens", type=int, default=0, help="give every request this many tokens")
+    ap.add_argument("--low-latency", action="store_true", help="batched resume with KVR_LOW_LATENCY")
     ap.add_argument("--no-extras", action="store_true", help="skip kernels-alone, lone-request and CPU legs")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -79,6 +79,8 @@ enum {
 
 /* call flags */
 #define KVR_SYNC 1u                  /* wait for the enqueued moves before returning */
+#define KVR_LOW_LATENCY 2u           /* batched resume, staged route: end a chunk wherever a request ends, so each
+                                        request is complete as soon as its own bytes are in (more, smaller launches) */
 /* pool flags (kvr_config.flags) */
 #define KVR_METADATA_ONLY 1u         /* bookkeeping only: no buffers, no CUDA calls, nothing moves */
 #define KVR_PROFILE 2u               /* bracket every mover launch with timing events (gather_ms, scatter_ms) */
@@ -206,7 +208,7 @@ kvr_status kvr_expire(kvr_pool *pool, const uint64_t *req, int32_t n, kvr_status
  * head (too few: KVR_HBM_FULL, unchanged), scatter the image into them (bytes
  * of a partial last block beyond n_tokens are not written), free the host
  * range, -> ACTIVE.  RETAINED: -> ACTIVE, same blocks, KVR_RESIDENT.  EXPIRED:
- * KVR_RECOMPUTE, unchanged.  ACTIVE: KVR_ERR_BAD_STATE.  flags: KVR_SYNC.
+ * KVR_RECOMPUTE, unchanged.  ACTIVE: KVR_ERR_BAD_STATE.  flags: KVR_SYNC, KVR_LOW_LATENCY.
  */
 kvr_status kvr_resume_from_host(kvr_pool *pool, const uint64_t *req, int32_t n, uint32_t flags, kvr_status *per_req);
 /*

@@ -143,6 +143,7 @@ struct kvr_pool {
   char *staging = nullptr;
   int *status_word = nullptr;             // pinned + mapped: movers write it, the host reads it
   BulkShape bulk{4, 4, 8192};
+  uint32_t call_flags = 0;                // flags of the call being served (set under the pool's lock)
   uint64_t copy_piece = 64ull << 20;      // largest single cudaMemcpyAsync of the staged route
   std::vector<cudaEvent_t> event_pool;
   std::map<uint64_t, Op> ops;
@@ -263,53 +264,44 @@ struct Plan {
   std::vector<int> req_chunk;     // item -> last chunk that holds bytes of it (-1: none)
 };
 
-// Chunk sizes of one staged move.  Every move starts with a small chunk and doubles up to the slot size: a
-// suspend's first copy over the link starts after a few microseconds of gathering, and the first requests of a
-// batched resume are complete (and usable) after milliseconds, not after a whole slot.  A resume also ends with
-// chunks that halve down to the small size, so little scattering is left after the last copy.  In between,
-// chunks are slot sized: few, large kernel launches.
-std::vector<uint64_t> chunk_caps(const kvr_pool *p, uint64_t total, bool ramp_down_too) {
+// Size limit of the next chunk of a staged move, given how many bytes earlier chunks hold and how many the move
+// has in all.  A chunk is never larger than everything before it (so sizes double from a small start: a suspend's
+// first copy over the link starts after a few microseconds of gathering, and the first requests of a batched
+// resume are complete after milliseconds), never larger than a slot, and, for a resume, never larger than half of
+// what is left (so sizes halve towards the end and little scattering remains after the last copy).
+uint64_t next_cap(const kvr_pool *p, uint64_t done, uint64_t total, bool ramp_down_too) {
   const uint64_t big = p->cfg.chunk_bytes;
   uint64_t small = 32ull << 20;
   if (small < (uint64_t)p->tile_bytes) small = align_up(p->tile_bytes, 4096);
   if (small > big) small = big;
-  std::vector<uint64_t> front, back;
-  uint64_t used = 0;
-  for (uint64_t c = small; used < total && c < big; c *= 2) {
-    front.push_back(c); used += c;
-    if (ramp_down_too && used < total) { back.push_back(c); used += c; }
+  uint64_t cap = done > small ? done : small;
+  if (ramp_down_too) {
+    const uint64_t left = total > done ? total - done : 0;
+    const uint64_t half = left / 2 > small ? left / 2 : small;
+    if (half < cap) cap = half;
   }
-  while (used < total) { front.push_back(big); used += big; }
-  // the largest chunk gives back what the ramps over-provision
-  if (!front.empty()) {
-    const uint64_t over = used - total;
-    uint64_t &largest = front.back();
-    if (over < largest && largest - over >= (uint64_t)p->tile_bytes) largest -= over;
-  }
-  std::vector<uint64_t> caps(front);
-  caps.insert(caps.end(), back.rbegin(), back.rend());
-  caps.push_back(small);      // chunks are cut on tile boundaries and may fall a little short: spare room
-  return caps;
+  if (cap > big) cap = big;
+  if (cap < (uint64_t)p->tile_bytes) cap = p->tile_bytes;
+  return cap;
 }
 
 // Staged route: cut the concatenated images into chunks on tile boundaries; chunk k goes to slot
-// (ring.next + k) mod slots and holds at most caps[k] bytes.
+// (ring.next + k) mod slots and holds at most next_cap() bytes.
 void plan_staged(kvr_pool *p, const std::vector<Item> &items, Ring &ring, bool ramp_down_too, const char *desc_dev, Plan &pl) {
   uint64_t total = 0;
   for (auto &it : items) total += (uint64_t)it.n_tokens * p->bpt;
-  const std::vector<uint64_t> caps = chunk_caps(p, total, ramp_down_too);
   const int nslots = (int)ring.slots.size();
   Chunk cur;
-  uint64_t fill = 0, cap = caps[0];
+  uint64_t fill = 0, done = 0, cap = 0;
   auto open = [&]() {
     cur = Chunk();
     cur.slot = (ring.next + (int)pl.chunks.size()) % nslots;
     cur.seg_begin = pl.segs.size();
     fill = 0;
-    cap = caps[pl.chunks.size() < caps.size() ? pl.chunks.size() : caps.size() - 1];
+    cap = next_cap(p, done, total, ramp_down_too);
   };
   auto flush = [&]() {
-    if (cur.nsegs) { cur.bytes = fill; pl.chunks.push_back(cur); }
+    if (cur.nsegs) { cur.bytes = fill; done += fill; pl.chunks.push_back(cur); }
     open();
   };
   open();
@@ -348,6 +340,9 @@ void plan_staged(kvr_pool *p, const std::vector<Item> &items, Ring &ring, bool r
       q0 = q1;
       if (cap - fill < (uint64_t)p->row) flush();
     }
+    // low-latency resume: close the chunk where a request ends, so the request is complete (its scatter launched)
+    // as soon as its own bytes have arrived instead of waiting for the rest of a slot
+    if (ramp_down_too && (p->call_flags & KVR_LOW_LATENCY) && T > 0 && cur.nsegs) flush();
   }
   flush();
 }
@@ -984,7 +979,10 @@ static kvr_status resume_common(kvr_pool *p, std::vector<Item> &items, uint64_t 
   uint64_t seq = 0;
   if (!p->meta_only && !items.empty()) {
     std::vector<uint64_t> none;
-    if (kvr_status s = enqueue(p, OP_RESUME, items, p->cfg.route, nullptr, block_tag, none, t_call, &seq)) return s;
+    p->call_flags = flags;
+    const kvr_status s = enqueue(p, OP_RESUME, items, p->cfg.route, nullptr, block_tag, none, t_call, &seq);
+    p->call_flags = 0;
+    if (s) return s;
   }
   for (auto &it : items) free_host(p, *it.r, seq);
   if (seq && (flags & KVR_SYNC)) return wait_ops(p, seq, 60000);

@@ -11,6 +11,7 @@ ERR_INVALID_ARG, ERR_UNKNOWN_REQUEST, ERR_BAD_STATE, ERR_GEOMETRY = -1, -2, -3, 
 ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM = -5, -6, -7
 ACTIVE, RETAINED, SUSPENDING, HOST, RESUMING, EXPIRED = 0, 1, 2, 3, 4, 5
 SYNC = 1
+LOW_LATENCY = 2
 METADATA_ONLY, PROFILE = 1, 2
 ROUTE_STAGED, ROUTE_MAPPED, ROUTE_DMA2D = 1, 2, 3
 LAYER_MAJOR, BLOCK_MAJOR = 0, 1

@@ -550,3 +550,26 @@ def test_a_wait_that_runs_out_is_reported_and_the_pool_stays_usable():
     assert a == b
     t.assert_same_pool()
     t.close()
+
+
+def test_low_latency_resume_completes_requests_one_by_one():
+    """Same bytes and bookkeeping with KVR_LOW_LATENCY; every request is complete as soon as its own bytes are in:
+    in order, the first long before the last, none later than under the default plan (where requests that share a
+    chunk finish together)."""
+    geom = (8, 8, 128, 2, 16)                      # 32 KiB per token
+    t = Twin(geom, 512, 256 << 20, seed=29, chunk_bytes=256 << 20)
+    ids = [0, 1, 2, 3]
+    for rid in ids:
+        assert t.both("admit", rid, 1500)[1][0] == kvr.OK        # 47 MiB each: all four fit one 256 MiB chunk
+    lat = {}
+    for flags in (0, kvr.LOW_LATENCY):
+        assert t.o.suspend_to_host(ids) == t.g.suspend_to_host(ids, kvr.SYNC)
+        assert t.o.resume_from_host(ids) == t.g.resume_from_host(ids, flags)
+        assert t.g.wait() == kvr.OK
+        lat[flags] = [t.g.latency(r)[2] for r in ids]
+        t.assert_same_pool()
+    for a, b in zip(lat[kvr.LOW_LATENCY], lat[0]):                   # never later than under the default plan
+        assert a <= 1.2 * b + 0.3
+    assert lat[kvr.LOW_LATENCY][0] < 0.5 * lat[kvr.LOW_LATENCY][3]   # one by one, in order
+    assert sorted(lat[kvr.LOW_LATENCY]) == lat[kvr.LOW_LATENCY]
+    t.close()
