@@ -320,6 +320,10 @@ def run_longctx(args):
             "resume_loss_pct_overlap_and_load": 100 * (1 - ovl_load["resume_gbs"] / seq["resume_gbs"]),
             "load_loss_pct": 100 * (1 - ovl_load["load_gbs"] / load_alone)},
         "host_link": link, "clocks": clocks,
+        "roofline": {"bound": "hbm", "peak": peak, "unit": "GB/s", "tile_bytes": BS * H * D * e,
+                     "gather_frac": 2 * st["gather_bytes"] / max(st["gather_ms"], 1e-9) / 1e6 / peak,
+                     "scatter_frac": 2 * st["scatter_bytes"] / max(st["scatter_ms"], 1e-9) / 1e6 / peak,
+                     "note": "CUDA events around every mover launch, all phases of this run"},
         "gpu_launches": int(st["gather_launches"] + st["scatter_launches"]),
     }
     print(json.dumps(out))

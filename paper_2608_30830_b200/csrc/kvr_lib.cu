@@ -503,6 +503,15 @@ kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> &items,
     p->st.desc_bytes += desc_bytes;
   }
 
+  // size of one link copy: 64 MiB, or more when the move is so large that 64 MiB pieces would put thousands of
+  // entries into the copy stream (a full stream queue blocks the caller, and with it the next call's overlap)
+  uint64_t piece = p->copy_piece;
+  {
+    uint64_t total = 0;
+    for (auto &ch : pl.chunks) total += ch.bytes;
+    const uint64_t floor_piece = align_up(total / 256 + 1, 1 << 20);
+    if (piece < floor_piece) piece = floor_piece;
+  }
   for (size_t ci = 0; ci < pl.chunks.size(); ++ci) {
     const Chunk &ch = pl.chunks[ci];
     cudaEvent_t cd;
@@ -522,8 +531,8 @@ kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> &items,
       // the copies go out in pieces: one very large cudaMemcpyAsync to pinned memory sustains less than the same
       // bytes in 64 MiB calls on some hosts (51.5 vs 56.3 GB/s measured), and never more
       for (auto &cp : ch.copies)
-        for (uint64_t o = 0; o < cp.bytes; o += p->copy_piece) {
-          const uint64_t n = cp.bytes - o < p->copy_piece ? cp.bytes - o : p->copy_piece;
+        for (uint64_t o = 0; o < cp.bytes; o += piece) {
+          const uint64_t n = cp.bytes - o < piece ? cp.bytes - o : piece;
           CU(cudaMemcpyAsync(p->h_arena + cp.lin_off + o, sl.ptr + cp.slot_off + o, n, cudaMemcpyDefault, c));
           p->st.d2h_copies++; p->st.d2h_bytes += n;
         }
@@ -532,8 +541,8 @@ kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> &items,
     } else {
       if (sl.used) CU(cudaStreamWaitEvent(c, sl.freed, 0));
       for (auto &cp : ch.copies)
-        for (uint64_t o = 0; o < cp.bytes; o += p->copy_piece) {
-          const uint64_t n = cp.bytes - o < p->copy_piece ? cp.bytes - o : p->copy_piece;
+        for (uint64_t o = 0; o < cp.bytes; o += piece) {
+          const uint64_t n = cp.bytes - o < piece ? cp.bytes - o : piece;
           CU(cudaMemcpyAsync(sl.ptr + cp.slot_off + o, p->h_arena + cp.lin_off + o, n, cudaMemcpyDefault, c));
           p->st.h2d_copies++; p->st.h2d_bytes += n;
         }
