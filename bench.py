@@ -535,7 +535,7 @@ def run_ours(args):
     if rank == 0:
         # kernels inside the timed region (profiling events around every launch)
         d = {k: s1[k] - s0[k] for k in ("gather_launches", "scatter_launches", "gather_bytes", "scatter_bytes",
-                                        "gather_ms", "scatter_ms", "d2h_bytes", "h2d_bytes", "desc_bytes",
+                                        "gather_ms", "scatter_ms", "gather_kernel_ms", "scatter_kernel_ms", "d2h_bytes", "h2d_bytes", "desc_bytes",
                                         "d2h_copies", "h2d_copies")}
         peak, peak_kind = peaks()
         g_gbs = 2 * d["gather_bytes"] / max(d["gather_ms"], 1e-9) / 1e6
@@ -554,6 +554,11 @@ def run_ours(args):
                     "algorithmic_bytes_per_launch": alg_per_launch,
                     "traffic": 0.979 * alg_per_launch,
                     "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum on a 1 GiB chunk, scaled by bytes per launch",
+                    "in_kernel": {
+                        "what": "the same launches timed by the kernels themselves: earliest CTA start to latest CTA end "
+                                "(%globaltimer), i.e. without the launch and completion latency the events include",
+                        "gather_frac": 2 * d["gather_bytes"] / max(d["gather_kernel_ms"], 1e-9) / 1e6 / peak,
+                        "scatter_frac": 2 * d["scatter_bytes"] / max(d["scatter_kernel_ms"], 1e-9) / 1e6 / peak},
                     "gather": {"gbs": g_gbs, "frac": g_gbs / peak, "launches": d["gather_launches"],
                                "avg_us": 1e3 * d["gather_ms"] / max(d["gather_launches"], 1)},
                     "scatter": {"gbs": s_gbs, "frac": s_gbs / peak, "launches": d["scatter_launches"],

@@ -136,7 +136,9 @@ typedef struct {
   uint64_t gather_bytes, scatter_bytes;          /* payload bytes moved by the kernels */
   uint64_t d2h_bytes, h2d_bytes;                 /* bytes moved by copies (descriptors excluded) */
   uint64_t desc_bytes;                           /* descriptor and block-table bytes uploaded */
-  double gather_ms, scatter_ms;                  /* summed kernel durations, KVR_PROFILE only */
+  double gather_ms, scatter_ms;                  /* summed kernel durations by CUDA events, KVR_PROFILE only */
+  double gather_kernel_ms, scatter_kernel_ms;    /* the same launches timed by the kernels themselves (first CTA
+                                                    start to last CTA end, %globaltimer), KVR_PROFILE only */
 } kvr_stats;
 
 /*

@@ -46,6 +46,12 @@ __device__ __forceinline__ void scan_segments(const MoveArgs &a, long long *cum)
   __syncthreads();
 }
 
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
 struct Tile {
   char *pool_ptr;   // first byte of the tile in the pool
   char *lin_ptr;    // first byte of the tile in the linear image
@@ -83,6 +89,7 @@ template <bool GATHER>
 __global__ void __launch_bounds__(kWarpThreads) move_warp_kernel(const MoveArgs a) {
   // (nsegs + 1) prefix sums, sized at launch (typically a few dozen bytes)
   extern __shared__ __align__(8) long long cum[];
+  if (a.stamp && threadIdx.x == 0) atomicMin(a.stamp, global_ns());
   scan_segments(a, cum);
   const int lane = threadIdx.x & 31;
   const int warps_per_cta = blockDim.x >> 5;
@@ -102,6 +109,7 @@ __global__ void __launch_bounds__(kWarpThreads) move_warp_kernel(const MoveArgs 
     }
     for (; i < nvec; i += 32) __stcs(dst + i, __ldcs(src + i));
   }
+  if (a.stamp && lane == 0) atomicMax(a.stamp + 1, global_ns());     // every warp: the latest one wins
 }
 
 // ---- bulk mover ----------------------------------------------------------------------
@@ -158,6 +166,7 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32) move_bulk_kernel(const Mov
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  if (a.stamp && threadIdx.x == 0) atomicMin(a.stamp, global_ns());
   if (lane == 0) {
     for (int s = 0; s < STAGES; ++s) mbar_init(smem_addr(&bars[warp][s]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -219,6 +228,7 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32) move_bulk_kernel(const Mov
     for (int s = 0; s < STAGES; ++s) mbar_wait(smem_addr(&bars[warp][s]), (phase_bits >> s) & 1u);
   }
   bulk_wait_all();
+  if (a.stamp) atomicMax(a.stamp + 1, global_ns());                  // every pipeline, after its last store landed
 }
 
 // Synthetic competing load: every CTA streams one 32 KiB slice of a large buffer and folds it into a sink word.

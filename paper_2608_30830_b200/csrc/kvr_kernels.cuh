@@ -33,6 +33,8 @@ struct MoveArgs {
   int row_bytes;         // kv_heads * head_dim * dtype_bytes (multiple of 16)
   int block_size;
   int *status;           // DEVICE: error word (0 = fine), written only when a bounded wait runs out
+  unsigned long long *stamp;  // DEVICE or NULL: stamp[0] = earliest start, stamp[1] = latest end of any CTA, in
+                              // %globaltimer nanoseconds (the host initialises them to ~0 and 0)
 };
 
 struct BulkShape {       // tuning of the bulk mover

@@ -89,6 +89,7 @@ struct Op {
   std::vector<ReqDone> reqs;                        // request -> index of the chunk that completes it (-1: none)
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof;   // kernel brackets (KVR_PROFILE)
   int desc = -1;
+  size_t stamp_off = 0; int n_stamps = 0;           // in-kernel time stamps inside the descriptor buffer (KVR_PROFILE)
   double host_ms = 0;
 };
 
@@ -196,6 +197,14 @@ void retire(kvr_pool *p, Op &op) {
       if (op.kind == OP_SUSPEND || op.kind == OP_EXPORT) p->st.gather_ms += ms; else p->st.scatter_ms += ms;
     }
     put_event(p, pr.first); put_event(p, pr.second);
+  }
+  if (op.desc >= 0 && op.n_stamps) {
+    // first CTA start to last CTA end of every launch, as the kernels stamped them
+    const unsigned long long *st = reinterpret_cast<const unsigned long long *>(p->descs[op.desc].h + op.stamp_off);
+    double ms = 0;
+    for (int i = 0; i < op.n_stamps; ++i)
+      if (st[2 * i + 1] > st[2 * i]) ms += (double)(st[2 * i + 1] - st[2 * i]) * 1e-6;
+    if (op.kind == OP_SUSPEND || op.kind == OP_EXPORT) p->st.gather_kernel_ms += ms; else p->st.scatter_kernel_ms += ms;
   }
   for (auto e : op.chunk_done) put_event(p, e);
   put_event(p, op.start); put_event(p, op.read_done); put_event(p, op.done);
@@ -368,11 +377,12 @@ void plan_direct(kvr_pool *p, const std::vector<Item> &items, char *lin_base, co
   if (cur.nsegs) pl.chunks.push_back(cur);
 }
 
-kvr_status launch(kvr_pool *p, bool gather, const Seg *segs_dev, const Chunk &c, cudaStream_t s, Op &op) {
+kvr_status launch(kvr_pool *p, bool gather, const Seg *segs_dev, const Chunk &c, cudaStream_t s, Op &op,
+                  unsigned long long *stamp) {
   MoveArgs a{};
   a.segs = segs_dev + c.seg_begin; a.nsegs = c.nsegs; a.total_tiles = c.tiles;
   a.pool = p->d_pool; a.plane_stride = p->plane_stride; a.block_stride = p->block_stride; a.tile_bytes = p->tile_bytes;
-  a.row_bytes = p->row; a.block_size = p->BS; a.status = p->status_word;
+  a.row_bytes = p->row; a.block_size = p->BS; a.status = p->status_word; a.stamp = stamp;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   if (p->profile) {
     kvr_status s0 = get_event(p, &e0); if (s0) return s0;
@@ -470,9 +480,17 @@ kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> &items,
     plan_direct(p, items, route == KVR_ROUTE_MAPPED ? p->arena_dev : lin_dev, nullptr, pl);
   }
   const size_t seg_off = align_up(bt_bytes, 64);
-  const size_t desc_bytes = seg_off + pl.segs.size() * sizeof(Seg);
+  const size_t stamp_off = align_up(seg_off + pl.segs.size() * sizeof(Seg), 64);
+  const int n_stamps = p->profile ? (int)pl.chunks.size() : 0;
+  const size_t desc_bytes = n_stamps ? stamp_off + 16 * (size_t)n_stamps : seg_off + pl.segs.size() * sizeof(Seg);
   if ((s = get_desc(p, desc_bytes ? desc_bytes : 64, &op.desc))) return s;
   DescBuf &db = p->descs[op.desc];
+  for (int i = 0; i < n_stamps; ++i) {
+    unsigned long long *st = reinterpret_cast<unsigned long long *>(db.h + stamp_off) + 2 * i;
+    st[0] = ~0ull; st[1] = 0;
+  }
+  op.stamp_off = stamp_off; op.n_stamps = n_stamps;
+  unsigned long long *stamps_dev = n_stamps ? reinterpret_cast<unsigned long long *>(db.d + stamp_off) : nullptr;
   for (auto &it : items) if (it.nb) memcpy(db.h + it.bt_off, it.blocks, (size_t)it.nb * 4);
   for (auto &sg : pl.segs) sg.bt = reinterpret_cast<const int32_t *>(db.d + reinterpret_cast<uintptr_t>(sg.bt));
   if (!pl.segs.empty()) memcpy(db.h + seg_off, pl.segs.data(), pl.segs.size() * sizeof(Seg));
@@ -518,14 +536,14 @@ kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> &items,
     if ((s = get_event(p, &cd))) return s;
     op.chunk_done.push_back(cd);
     if (!staged) {
-      if ((s = launch(p, to_linear, segs_dev, ch, k, op))) return s;
+      if ((s = launch(p, to_linear, segs_dev, ch, k, op, stamps_dev ? stamps_dev + 2 * ci : nullptr))) return s;
       CU(cudaEventRecord(cd, k));
       continue;
     }
     Slot &sl = ring->slots[ch.slot];
     if (to_linear) {
       if (sl.used) CU(cudaStreamWaitEvent(k, sl.freed, 0));
-      if ((s = launch(p, true, segs_dev, ch, k, op))) return s;
+      if ((s = launch(p, true, segs_dev, ch, k, op, stamps_dev ? stamps_dev + 2 * ci : nullptr))) return s;
       CU(cudaEventRecord(sl.filled, k));
       CU(cudaStreamWaitEvent(c, sl.filled, 0));
       // the copies go out in pieces: one very large cudaMemcpyAsync to pinned memory sustains less than the same
@@ -548,7 +566,7 @@ kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> &items,
         }
       CU(cudaEventRecord(sl.filled, c));
       CU(cudaStreamWaitEvent(k, sl.filled, 0));
-      if ((s = launch(p, false, segs_dev, ch, k, op))) return s;
+      if ((s = launch(p, false, segs_dev, ch, k, op, stamps_dev ? stamps_dev + 2 * ci : nullptr))) return s;
       CU(cudaEventRecord(sl.freed, k));
       CU(cudaEventRecord(cd, k));
     }
@@ -566,6 +584,8 @@ kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> &items,
   } else {
     CU(cudaEventRecord(op.read_done, reader));
   }
+  if (n_stamps)      // the stamps come back with the move: `last` is ordered after every launch
+    CU(cudaMemcpyAsync(db.h + stamp_off, db.d + stamp_off, 16 * (size_t)n_stamps, cudaMemcpyDeviceToHost, last));
   CU(cudaEventRecord(op.done, last));
 
   register_op(p, op, items, pl.req_chunk, kind, t_call, out_seq);

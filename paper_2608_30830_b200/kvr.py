@@ -63,7 +63,7 @@ class Stats(C.Structure):
                [(n, C.c_int64) for n in ("ops_in_flight", "gather_launches", "scatter_launches",
                                          "d2h_copies", "h2d_copies")] + \
                [(n, C.c_uint64) for n in ("gather_bytes", "scatter_bytes", "d2h_bytes", "h2d_bytes", "desc_bytes")] + \
-               [(n, C.c_double) for n in ("gather_ms", "scatter_ms")]
+               [(n, C.c_double) for n in ("gather_ms", "scatter_ms", "gather_kernel_ms", "scatter_kernel_ms")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}

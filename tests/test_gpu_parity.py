@@ -265,6 +265,8 @@ def test_tiny_config_full_size():
     s = t.g.stats()
     assert s["bytes_suspended"] == s["bytes_resumed"] == int(lens.sum()) * 32768
     assert s["gather_ms"] > 0 and s["scatter_ms"] > 0
+    # the kernels' own stamps: a positive time, shorter than what the events around the launches saw
+    assert 0 < s["gather_kernel_ms"] < s["gather_ms"] and 0 < s["scatter_kernel_ms"] < s["scatter_ms"]
     t.close()
 
 
