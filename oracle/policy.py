@@ -15,7 +15,6 @@ cheaper branch.
 Pins (tests): the cross-platform table's t_1 / t*, the load-sweep table's exact entries (0.020 at half the critical
 load) and its fixed-timer columns against the closed form beta_2 P(W <= T) + beta_3 P(W > T).
 """
-import heapq
 import math
 
 
@@ -42,24 +41,28 @@ def t2(lam, c2, w_ref, beta2, beta3):
 
 
 def replay(arrivals, waits, c2, ttl, beta2, beta3):
-    """Mean GPU opportunity cost per request and the fraction resumed from a host copy.
-    arrivals must be non-decreasing.  ttl may be math.inf (host-retain)."""
-    departures = []                 # min-heap of times at which admitted contexts leave their slot
+    """Mean GPU opportunity cost per request and the fraction resumed from a host copy (Appendix D, replay rules).
+    arrivals must be non-decreasing.  ttl may be math.inf (host-retain).
+
+    The host tier is a plain list with one entry per occupied slot: the time at which that resident leaves.
+    Readings of the two ties the paper does not spell out: a resident whose departure falls exactly on an
+    arrival has left (its slot is free for that arrival), and a wait exactly equal to the timer resumes in time
+    (the copy is still there: beta_2)."""
+    occupied = []                   # departure times of the residents, in order of admission
     total = 0.0
     from_host = 0
     for a, w in zip(arrivals, waits):
         a, w = float(a), float(w)
-        while departures and departures[0] <= a:
-            heapq.heappop(departures)
-        if len(departures) < c2:                    # a slot is free: admitted
-            heapq.heappush(departures, a + min(w, ttl))
-            if w <= ttl:                            # resumes before the timer fires
-                total += beta2
-                from_host += 1
-            else:
-                total += beta3                      # expired: recompute at resume
+        # residents leave at their resume or when their one-shot timer fires; nobody is ever displaced
+        occupied = [leave for leave in occupied if leave > a]
+        admitted = len(occupied) < c2               # admission iff a host slot is free at the arrival
+        if admitted:
+            occupied.append(a + min(w, ttl))        # the slot is held until min(wait, timer)
+        if admitted and w <= ttl:
+            total += beta2                          # the resume finds its host copy
+            from_host += 1
         else:
-            total += beta3                          # not admitted: recompute at resume
+            total += beta3                          # timer fired first, or never admitted: recompute
     n = len(arrivals)
     return total / n, from_host / n
 

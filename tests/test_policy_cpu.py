@@ -94,6 +94,31 @@ def test_replay_small_case_by_hand():
     assert cost == pytest.approx((1 + 1 + 100 + 1 + 100) / 5) and frac == pytest.approx(3 / 5)
 
 
+def test_replay_ties_by_hand():
+    # one slot, a 10 s timer.  The two ties the paper leaves open, each worked by hand:
+    #  * r0 (arrives 0, waits 4) leaves at 4.0; r1 arrives at exactly 4.0 -> the slot is free for it: admitted;
+    #  * r1 waits exactly 10.0 = the timer -> it resumes in time: beta_2, and holds the slot until 14.0;
+    #  * r2 arrives at 13.0 while r1 still holds the slot -> not admitted: beta_3;
+    #  * r3 arrives at exactly 14.0 = r1's departure -> admitted; it waits 10.5 > timer -> expired at 24: beta_3;
+    #  * r4 arrives at 24.0 = the instant r3's timer fired -> admitted, waits 1: beta_2.
+    arr = [0.0, 4.0, 13.0, 14.0, 24.0]
+    w = [4.0, 10.0, 1.0, 10.5, 1.0]
+    cost, frac = policy.replay(arr, w, 1, 10.0, 1.0, 100.0)
+    assert cost == pytest.approx((1 + 1 + 100 + 100 + 1) / 5) and frac == pytest.approx(3 / 5)
+    # the same arrivals one tick earlier find the slot still taken
+    eps = 1e-9
+    cost, frac = policy.replay([0.0, 4.0 - eps, 13.0, 14.0, 24.0], w, 1, 10.0, 1.0, 100.0)
+    # r1 rejected (beta_3); r2 at 13 finds the slot free (r0 left at 4): beta_2, leaves at 14 -> r3 admitted as before
+    assert cost == pytest.approx((1 + 100 + 1 + 100 + 1) / 5) and frac == pytest.approx(3 / 5)
+
+
+def test_replay_capacity_zero_and_empty_tier():
+    # no host slots: everything recomputes; unlimited slots and no timer: everything resumes from host
+    arr, w = [0.0, 1.0, 2.0], [5.0, 5.0, 5.0]
+    assert policy.replay(arr, w, 0, math.inf, 1.0, 100.0) == (100.0, 0.0)
+    assert policy.replay(arr, w, 3, math.inf, 1.0, 100.0) == (1.0, 1.0)
+
+
 # ---- the library's policy functions against the oracle ---------------------------------------
 
 def test_library_policy_matches_oracle():
@@ -114,6 +139,9 @@ def test_library_policy_matches_oracle():
             branch, cr, ct, t2v = kvr.policy_select(prices, arr, w, mult * LCRIT, C2, WREF)
             ob, ocr, oct_, ot2 = policy.select_branch(arr, w, mult * LCRIT, C2, WREF, B2, B3)
             assert (branch, t2v) == (ob, ot2) and cr == pytest.approx(ocr, rel=1e-12) and ct == pytest.approx(oct_, rel=1e-12)
+    # the tie readings (departure exactly at an arrival; wait exactly equal to the timer)
+    arr, w = [0.0, 4.0, 13.0, 14.0, 24.0], [4.0, 10.0, 1.0, 10.5, 1.0]
+    assert kvr.policy_replay((1.0, 1.0, 100.0), arr, w, 1, 10.0) == pytest.approx(policy.replay(arr, w, 1, 10.0, 1.0, 100.0), rel=1e-12)
     with pytest.raises(kvr.KvrError):
         kvr.policy_break_evens(0.0, B2, B3)
     with pytest.raises(kvr.KvrError):
