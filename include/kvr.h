@@ -246,6 +246,12 @@ kvr_status kvr_import_from_device(kvr_pool *pool, const uint64_t *req, int32_t n
  *   block_table : HOST, nb = ceil(n_tokens / block_size) ids in [0, num_blocks)
  *   dst_device  : DEVICE, n_tokens * kvr_bytes_per_token(g) bytes, 16-byte aligned
  *   stream      : cudaStream_t (NULL = default stream); the work is enqueued, not waited for
+ * block_table may be pageable or page-locked: it is read only during the call (it is copied to a fixed host-side
+ * twin of the array, range-checked there and uploaded from there), so the caller may change or free it as soon
+ * as the call returns.  That upload comes from pageable memory, so the call can block the host until the work
+ * already queued on `stream` has finished (for instance the previous call's gather).
+ * A geometry whose tile (block_size x kv_heads x head_dim x dtype_bytes) exceeds 1 GiB is KVR_ERR_GEOMETRY, as in
+ * kvr_pool_create.
  * Runs on the current device.  The first call on each device looks up the array's address; make that
  * call before starting any stream capture.  All calls share the array: calls whose GPU work may overlap
  * (different streams or threads) race on it -- keep them on one stream or wait in between.  Nothing in

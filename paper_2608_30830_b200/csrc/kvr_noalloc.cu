@@ -15,6 +15,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "../../include/kvr.h"
 #include "kvr_kernels.cuh"
@@ -29,6 +30,13 @@ constexpr size_t kScratchBytes = kSegBytes + sizeof(int32_t) * (size_t)KVR_NOALL
 // Scratch of the allocation-free entry point.  In host code this name is only a handle for
 // cudaGetSymbolAddress(): it is not a device address and must never be passed to a kernel as is.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
+
+// Host-side twin of the array: the record and the table are first copied here, checked here, and uploaded from
+// here.  It is ordinary pageable memory, so the runtime has taken its own copy of it by the time each
+// cudaMemcpyAsync returns; the caller's table (pageable or page-locked) is read only during the call, and the ids
+// the kernel sees are exactly the ids that were range-checked.  g_stage_mu serialises the host side of calls.
+alignas(256) unsigned char g_stage[kScratchBytes];
+std::mutex g_stage_mu;
 
 constexpr int kMaxDevices = 64;
 unsigned char *g_scratch_ptr[kMaxDevices];   // device address of the array, per device ordinal (set up on first use)
@@ -73,8 +81,10 @@ extern "C" kvr_status kvr_gather_noalloc(const void *device_pool, const kvr_geom
   }
   if ((n_tokens + g->block_size - 1) / g->block_size != nb)
     return fail_na(KVR_ERR_INVALID_ARG, "nb must equal ceil(n_tokens / block_size)");
-  for (int32_t i = 0; i < nb; ++i)
-    if (block_table[i] < 0 || block_table[i] >= num_blocks) return fail_na(KVR_ERR_INVALID_ARG, "block id out of range");
+  // sizes in 64 bits: a tile is at most 1 GiB (the same rule as kvr_pool_create), so the kernel's int fields hold
+  const uint64_t row = bpt / 2 / (uint64_t)g->layers;
+  const uint64_t tile = row * (uint64_t)g->block_size;
+  if (tile > (1ull << 30)) return fail_na(KVR_ERR_GEOMETRY, "one tile exceeds 1 GiB");
   if (nb == 0) return KVR_OK;
 
   int dev = -1;
@@ -84,7 +94,6 @@ extern "C" kvr_status kvr_gather_noalloc(const void *device_pool, const kvr_geom
   unsigned char *scratch = g_scratch_ptr[dev];
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-  const int row = (int)(bpt / 2 / g->layers);
   kvr::Seg seg{};
   seg.bt = reinterpret_cast<const int32_t *>(scratch + kSegBytes);
   seg.img = static_cast<char *>(dst_device);
@@ -92,26 +101,33 @@ extern "C" kvr_status kvr_gather_noalloc(const void *device_pool, const kvr_geom
   seg.tile_begin = 0;
   seg.tile_count = 2ll * g->layers * nb;
   seg.nb = nb;
-  // Both copies read pageable host memory: the runtime stages such copies before returning, so the
-  // caller's table and this stack record may be reused as soon as the call returns.  They are ordered on
-  // `stream` before the kernel, and after whatever that stream ran before (e.g. the previous call).
-  cudaError_t e = cudaMemcpyAsync(scratch, &seg, sizeof seg, cudaMemcpyHostToDevice, st);
-  if (e == cudaSuccess)
-    e = cudaMemcpyAsync(scratch + kSegBytes, block_table, sizeof(int32_t) * (size_t)nb, cudaMemcpyHostToDevice, st);
-  if (e != cudaSuccess) return fail_na(KVR_ERR_CUDA, cudaGetErrorString(e));
+
+  {
+    std::lock_guard<std::mutex> hold(g_stage_mu);
+    int32_t *table = reinterpret_cast<int32_t *>(g_stage + kSegBytes);
+    memcpy(g_stage, &seg, sizeof seg);
+    memcpy(table, block_table, sizeof(int32_t) * (size_t)nb);
+    for (int32_t i = 0; i < nb; ++i)
+      if (table[i] < 0 || table[i] >= num_blocks) return fail_na(KVR_ERR_INVALID_ARG, "block id out of range");
+    // One upload of record + table from the pageable twin: the runtime copies a pageable source out before the call
+    // returns (after waiting for whatever `stream` ran before), so the twin is free again when the lock drops.  The
+    // upload is ordered on `stream` before the kernel and after the previous call's kernel.
+    cudaError_t e = cudaMemcpyAsync(scratch, g_stage, kSegBytes + sizeof(int32_t) * (size_t)nb, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return fail_na(KVR_ERR_CUDA, cudaGetErrorString(e));
+  }
 
   kvr::MoveArgs a{};
   a.segs = reinterpret_cast<const kvr::Seg *>(scratch);
   a.nsegs = 1;
   a.total_tiles = seg.tile_count;
   a.pool = static_cast<char *>(const_cast<void *>(device_pool));
-  a.tile_bytes = row * g->block_size;
-  a.plane_stride = (long long)num_blocks * a.tile_bytes;   // layer-major pool
-  a.block_stride = a.tile_bytes;
-  a.row_bytes = row;
+  a.tile_bytes = (int)tile;
+  a.plane_stride = (long long)num_blocks * (long long)tile;   // layer-major pool
+  a.block_stride = (long long)tile;
+  a.row_bytes = (int)row;
   a.block_size = g->block_size;
   a.status = nullptr;               // the warp mover has no bounded waits and never writes it
-  e = kvr::launch_move_warp(true, a, 0, g_sm_count[dev], st);
+  cudaError_t e = kvr::launch_move_warp(true, a, 0, g_sm_count[dev], st);
   if (e != cudaSuccess) return fail_na(KVR_ERR_CUDA, cudaGetErrorString(e));
   return KVR_OK;
 }
