@@ -1,8 +1,13 @@
 """The benchmark configurations at full size on the GPU, in the launch configuration bench.py times
 (staged route, default mover and chunk sizes).
 
-A host mirror of a 64-128 GiB pool does not exist, so parity is shown three ways:
+A host mirror of a 64-128 GiB pool does not exist, so parity is shown four ways:
   * bookkeeping (statuses, block tables, arena offsets, free queue) against a data-less oracle pool, call by call;
+  * EVERY image byte: the image, by definition, is image[plane][t] = pool[plane][table[t / BS]][t % BS]; that
+    expression is evaluated on the device with torch indexing (pinned once against the oracle's gather on a small
+    pool, below) and compared with the whole image the library wrote, request by request, after the suspend under
+    the old tables and after the resume under the new ones; and every pool row outside the resumed requests' valid
+    slots is shown unchanged through per-row checksums taken before and after;
   * sampled token rows: the oracle names, one by one, the pool byte offset and the image byte offset of a sampled
     (request, layer, plane, token); the bytes found there on the device / in the pinned arena must be equal;
   * one whole request: its blocks are read back into a small relabelled host pool, the oracle gathers that pool
@@ -109,11 +114,47 @@ class Rig:
         mini = self.dev.view(2 * L, self.NB, tile).index_select(1, blocks).cpu().numpy().reshape(-1)
         return orc.gather(mini, L, H, D, e, BS, d["nb"], np.arange(d["nb"]), d["n_tokens"])
 
+    def row_sums(self):
+        """One wrapping int64 sum per pool row (one token slot of one plane of one block): shape (2L, NB, BS)."""
+        L, H, D, e, BS = self.geom
+        return self.dev.view(torch.int64).view(2 * L * self.NB * BS, self.row // 8).sum(dim=1).view(2 * L, self.NB, BS)
+
+    def image_by_definition(self, table, n, p0, p1):
+        """Planes [p0, p1) of the image of a request with this table and n tokens, from the pool as it is now."""
+        return image_by_definition(self.dev, self.geom, self.NB, table, n, p0, p1)
+
+    def assert_whole_images(self, ids, tables, images, slab_bytes=1 << 30):
+        """Every byte of every image (numpy views of the pinned arena) against the definition under `tables`."""
+        L, H, D, e, BS = self.geom
+        for rid in ids:
+            n = int(self.o.info(rid)[1]["n_tokens"])
+            if n == 0:
+                continue
+            img = torch.from_numpy(images[rid]).view(2 * L, n, self.row)
+            step = max(1, slab_bytes // (n * self.row))
+            for p0 in range(0, 2 * L, step):
+                p1 = min(2 * L, p0 + step)
+                want = self.image_by_definition(tables[rid], n, p0, p1)
+                got = img[p0:p1].cuda()
+                assert torch.equal(got, want), "image of request %d differs in planes %d..%d" % (rid, p0, p1)
+                del want, got
+
     def close(self):
         self.g.close()
         self.o.close()
         del self.rows, self.dev
         cleanup()
+
+
+def image_by_definition(dev_pool, geom, NB, table, n, p0=0, p1=None):
+    """image[plane][t][:] = pool[plane][table[t // BS]][t % BS][:] for planes [p0, p1), as a (planes, n, row) uint8
+    tensor on the device: the definition of the host image, written with torch indexing (layer-major pool)."""
+    L, H, D, e, BS = geom
+    row = H * D * e
+    p1 = 2 * L if p1 is None else p1
+    blocks = torch.as_tensor(np.asarray(table, dtype=np.int64), device=dev_pool.device)
+    tiles = dev_pool.view(2 * L, NB, BS * row)[p0:p1].index_select(1, blocks)          # (planes, nb, tile)
+    return tiles.reshape(p1 - p0, len(table) * BS, row)[:, :n]
 
 
 def untouched_rows(rig, ids, others, k=256):
@@ -139,15 +180,35 @@ def untouched_rows(rig, ids, others, k=256):
     return out
 
 
+def touched_mask(rig, ids):
+    """(NB, BS) bool: the token slots a resume of `ids` writes (valid slots of their current blocks)."""
+    BS = rig.geom[4]
+    mask = torch.zeros(rig.NB, BS, dtype=torch.bool)
+    for rid in ids:
+        d = rig.o.info(rid)[1]
+        n, blocks = int(d["n_tokens"]), d["blocks"].astype(np.int64)
+        if n == 0:
+            continue
+        mask[torch.from_numpy(blocks[:n // BS])] = True
+        if n % BS:
+            mask[int(blocks[-1]), :n % BS] = True
+    return mask.cuda()
+
+
 def suspend_resume_checked(rig, ids, whole=None, k=1536, others=()):
     samples = rig.sample(ids, k)
     before = rig.read_pool_rows(samples)
     want_whole = rig.whole_request_image(whole) if whole is not None else None
+    sums0 = rig.row_sums()
+    old_tables = {rid: rig.o.info(rid)[1]["blocks"].copy() for rid in ids}
     st, per = rig.both("suspend_to_host", ids)
     assert st == kvr.OK
     assert rig.g.wait() == kvr.OK, kvr.last_error()
     assert np.array_equal(rig.read_image_rows(samples), before)           # image rows = the oracle-addressed pool rows
     assert np.array_equal(rig.read_pool_rows(samples), before)            # the suspend left the pool alone
+    assert torch.equal(rig.row_sums(), sums0)                             # ... every row of it
+    images = {rid: rig.g.host_image(rid) for rid in ids}                  # views of the arena; they outlive the resume
+    rig.assert_whole_images(ids, old_tables, images)                      # every image byte, by definition
     if whole is not None:
         assert np.array_equal(rig.g.host_image(whole), want_whole)
     for rid in ids:
@@ -166,9 +227,33 @@ def suspend_resume_checked(rig, ids, whole=None, k=1536, others=()):
         assert rig.o.info(rid)[1]["blocks"].tolist() == rig.g.info(rid)[1]["blocks"].tolist()
     after = rig.resample_pool_offsets(samples)
     assert np.array_equal(rig.read_pool_rows(after), before)              # same logical rows under the new tables
+    new_tables = {rid: rig.o.info(rid)[1]["blocks"].copy() for rid in ids}
+    rig.assert_whole_images(ids, new_tables, images)                      # every byte landed where the new tables say
+    same = rig.row_sums() == sums0                                        # and nothing else in the pool changed
+    assert bool((same | touched_mask(rig, ids).unsqueeze(0)).all()), "a row outside the resumed requests changed"
+    del same, sums0
     if whole is not None:
         assert np.array_equal(rig.whole_request_image(whole), want_whole)
     assert rig.o.free_queue().tolist() == rig.g.free_queue().tolist()
+
+
+def test_definition_on_the_device_equals_the_oracle_gather():
+    """Pins image_by_definition (the torch expression the full-size checks rely on) to the oracle, element by
+    element, on a pool small enough to mirror on the host: ragged length, shuffled table, several planes."""
+    geom = (3, 2, 64, 2, 4)
+    L, H, D, e, BS = geom
+    NB = 96
+    rng = np.random.default_rng(5)
+    host_pool = rng.integers(0, 256, size=NB * BS * 2 * L * H * D * e, dtype=np.uint8)
+    dev_pool = torch.from_numpy(host_pool).cuda()
+    for n in (1, 4, 37, 40, 163):
+        nb = -(-n // BS)
+        table = rng.permutation(NB)[:nb].astype(np.int32)
+        want = orc.gather(host_pool, L, H, D, e, BS, NB, table, n)
+        got = image_by_definition(dev_pool, geom, NB, table, n).cpu().numpy().reshape(-1)
+        assert np.array_equal(got, want), n
+        part = image_by_definition(dev_pool, geom, NB, table, n, 2, 5).cpu().numpy().reshape(-1)
+        assert np.array_equal(part, want.reshape(2 * L, -1)[2:5].reshape(-1))
 
 
 def test_config2_llama3_8b_shaped_full_size():
@@ -243,9 +328,14 @@ def test_config5_long_context_overlapped_suspend_and_resume():
     out_first, stay = ids[:half], ids[half:]
     s_out = rig.sample(out_first, 512)
     rows_out = rig.read_pool_rows(s_out)
+    sums0 = rig.row_sums()
+    tables = {rid: rig.o.info(rid)[1]["blocks"].copy() for rid in ids}
     assert rig.both("suspend_to_host", out_first)[0] == kvr.OK             # phase A (untimed): one half on the host
     assert rig.g.wait() == kvr.OK
     assert np.array_equal(rig.read_image_rows(s_out), rows_out)
+    assert torch.equal(rig.row_sums(), sums0)
+    images = {rid: rig.g.host_image(rid) for rid in out_first}
+    rig.assert_whole_images(out_first, tables, images)                     # every byte of the first half's images
     s_stay = rig.sample(stay, 512)
     rows_stay = rig.read_pool_rows(s_stay)
     # phase B: both directions at once
@@ -256,8 +346,25 @@ def test_config5_long_context_overlapped_suspend_and_resume():
     assert np.array_equal(rig.read_pool_rows(rig.resample_pool_offsets(s_out)), rows_out)
     for rid in out_first:
         assert rig.o.info(rid)[1]["blocks"].tolist() == rig.g.info(rid)[1]["blocks"].tolist()
+    # the overlapped pair, completely: the second half's images under the tables they had (their blocks were freed,
+    # and the overlapped resume took blocks from the head of the queue, i.e. other ones: see the assert), and the
+    # first half under its new tables; every other row unchanged
+    new_out = {rid: rig.o.info(rid)[1]["blocks"].copy() for rid in out_first}
+    taken = set(int(b) for rid in out_first for b in new_out[rid])
+    images.update({rid: rig.g.host_image(rid) for rid in stay})
+    if not taken & set(int(b) for rid in stay for b in tables[rid]):
+        rig.assert_whole_images(stay, tables, images)
+    rig.assert_whole_images(out_first, new_out, images)
+    same = rig.row_sums() == sums0
+    assert bool((same | touched_mask(rig, out_first).unsqueeze(0)).all())
+    del same
     assert rig.both("resume_from_host", stay)[0] == kvr.OK
     assert rig.g.wait() == kvr.OK
     assert np.array_equal(rig.read_pool_rows(rig.resample_pool_offsets(s_stay)), rows_stay)
+    new_stay = {rid: rig.o.info(rid)[1]["blocks"].copy() for rid in stay}
+    rig.assert_whole_images(stay, new_stay, images)
+    same = rig.row_sums() == sums0
+    assert bool((same | touched_mask(rig, ids).unsqueeze(0)).all())
+    del same, sums0
     check_invariants(rig.g, ids)
     rig.close()
