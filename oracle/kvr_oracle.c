@@ -17,10 +17,11 @@ typedef struct {
   uint64_t id;
   int32_t state;
   int64_t n_tokens;
-  int32_t nb;
-  int32_t *blocks;        /* ACTIVE / RETAINED */
-  uint8_t *image;         /* HOST (with_data) */
-  uint64_t image_bytes;   /* n_tokens * bytes_per_token */
+  int32_t nb;             /* ceil(n_tokens / BS): logical blocks, shared prefix included */
+  int32_t n_shared;       /* leading blocks that are a shared prefix (whole blocks, never moved) */
+  int32_t *blocks;        /* ACTIVE / RETAINED: all nb entries; HOST: the n_shared prefix entries it still refers to */
+  uint8_t *image;         /* HOST (with_data): the private suffix, tokens [n_shared*BS, n_tokens) */
+  uint64_t image_bytes;   /* (n_tokens - n_shared*BS) * bytes_per_token */
   uint64_t arena_off;     /* HOST */
   uint64_t arena_len;     /* image_bytes rounded up to ARENA_ALIGN */
 } orc_req;
@@ -35,6 +36,7 @@ struct orc_pool {
   uint64_t data_bytes;
   int32_t *freeq;          /* freeq[0] is the head */
   int64_t n_free;
+  int32_t *refcnt;         /* per block: how many (request, position) references name it; 0 <=> in the free queue */
   orc_req *reqs;
   int64_t n_reqs, cap_reqs;
   orc_range *used;         /* host ranges in use, sorted by offset */
@@ -146,10 +148,12 @@ orc_pool *orc_pool_create(int32_t L, int32_t H, int32_t D, int32_t e, int32_t BS
     for (int32_t i = 0; i < NB; ++i) p->freeq[i] = i;
   }
   p->n_free = NB;
+  p->refcnt = (int32_t *)calloc((size_t)NB, sizeof(int32_t));
+  if (!p->refcnt) { free(p->freeq); free(p); return NULL; }
   if (with_data) {
     p->data_bytes = (uint64_t)NB * (uint64_t)BS * p->bpt;
     p->data = (uint8_t *)calloc((size_t)p->data_bytes, 1);
-    if (!p->data) { free(p->freeq); free(p); return NULL; }
+    if (!p->data) { free(p->refcnt); free(p->freeq); free(p); return NULL; }
   }
   return p;
 }
@@ -157,7 +161,7 @@ orc_pool *orc_pool_create(int32_t L, int32_t H, int32_t D, int32_t e, int32_t BS
 void orc_pool_destroy(orc_pool *p) {
   if (!p) return;
   for (int64_t i = 0; i < p->n_reqs; ++i) { free(p->reqs[i].blocks); free(p->reqs[i].image); }
-  free(p->reqs); free(p->used); free(p->freeq); free(p->data); free(p);
+  free(p->reqs); free(p->used); free(p->freeq); free(p->refcnt); free(p->data); free(p);
 }
 
 uint8_t *orc_pool_data(orc_pool *p) { return p ? p->data : NULL; }
@@ -231,9 +235,29 @@ static void drop_host_copy(orc_pool *p, orc_req *r) {
   r->arena_off = 0; r->arena_len = 0;
 }
 
+/* take one reference on each id (a block popped from the free queue starts at 1) */
+static void ref_blocks(orc_pool *p, const int32_t *ids, int32_t n) {
+  for (int32_t i = 0; i < n; ++i) p->refcnt[ids[i]] += 1;
+}
+
+/* give up the references blocks[from .. to) of a request, in logical order; a block whose last
+ * reference goes joins the free-queue tail (Appendix A: released blocks return to the eviction tail) */
+static void unref_blocks(orc_pool *p, const int32_t *blocks, int32_t from, int32_t to) {
+  for (int32_t i = from; i < to; ++i) {
+    p->refcnt[blocks[i]] -= 1;
+    if (p->refcnt[blocks[i]] == 0) freeq_push(p, &blocks[i], 1);
+  }
+}
+
+/* the request lets go of every block it refers to */
 static void drop_blocks(orc_pool *p, orc_req *r) {
-  freeq_push(p, r->blocks, r->nb);
+  int32_t held = (r->state == ORC_HOST) ? r->n_shared : r->nb;
+  unref_blocks(p, r->blocks, 0, held);
   free(r->blocks); r->blocks = NULL;
+}
+
+static int64_t private_tokens(const orc_pool *p, const orc_req *r) {
+  return r->n_tokens - (int64_t)r->n_shared * p->BS;
 }
 
 /* batch result: the most negative status if any is an error, else the largest */
@@ -268,8 +292,67 @@ int32_t orc_request_admit(orc_pool *p, uint64_t id, int64_t n_tokens, int32_t *o
   r->n_tokens = n_tokens;
   r->nb = nb;
   r->image_bytes = (uint64_t)n_tokens * p->bpt;
+  r->n_shared = 0;
   r->blocks = (int32_t *)malloc(sizeof(int32_t) * (size_t)(nb ? nb : 1));
   freeq_pop(p, nb, r->blocks);
+  ref_blocks(p, r->blocks, nb);
+  if (out_blocks) memcpy(out_blocks, r->blocks, sizeof(int32_t) * (size_t)nb);
+  return ORC_OK;
+}
+
+/* Admission that shares a prefix (Section 2, approval-gated workload: the shared system prefix is reused through
+ * prefix caching, "so only the private suffix contributes per-request suspended state").  The new request's first
+ * n_shared logical blocks ARE the donor's first n_shared blocks (one more reference each); the rest come from the
+ * free-queue head.  Readings (the paper names no mechanism): sharing is by whole blocks -- n_shared*BS tokens must
+ * lie inside both the new request and the donor; the donor may be in any state in which it still refers to those
+ * blocks (ACTIVE / RETAINED: any of its full blocks; HOST: its own shared prefix). */
+int32_t orc_request_admit_sharing(orc_pool *p, uint64_t id, int64_t n_tokens, uint64_t donor_id, int32_t n_shared,
+                                  int32_t *out_blocks, int32_t cap) {
+  if (!p || n_tokens < 0 || n_shared < 0) return ORC_ERR_INVALID_ARG;
+  int64_t nb64 = (n_tokens + p->BS - 1) / p->BS;
+  if ((int64_t)n_shared * p->BS > n_tokens) return ORC_ERR_INVALID_ARG;
+  if (out_blocks && (int64_t)cap < nb64) return ORC_ERR_INVALID_ARG;
+  orc_req *r = find_req(p, id);
+  if (r && r->state != ORC_EXPIRED) return ORC_ERR_BAD_STATE;
+  int32_t *prefix = NULL;
+  if (n_shared > 0) {
+    if (donor_id == id) return ORC_ERR_INVALID_ARG;
+    orc_req *d = find_req(p, donor_id);
+    if (!d) return ORC_ERR_UNKNOWN_REQUEST;
+    if (d->state == ORC_ACTIVE || d->state == ORC_RETAINED) {
+      if ((int64_t)n_shared * p->BS > d->n_tokens) return ORC_ERR_INVALID_ARG;
+    } else if (d->state == ORC_HOST) {
+      if (n_shared > d->n_shared) return ORC_ERR_INVALID_ARG;
+    } else {
+      return ORC_ERR_BAD_STATE;            /* a discarded donor refers to nothing */
+    }
+    prefix = (int32_t *)malloc(sizeof(int32_t) * (size_t)n_shared);
+    if (!prefix) return ORC_ERR_NOMEM;
+    memcpy(prefix, d->blocks, sizeof(int32_t) * (size_t)n_shared);
+  }
+  if (nb64 - n_shared > p->n_free) { free(prefix); p->st.hbm_full_rejects++; return ORC_HBM_FULL; }
+  int32_t nb = blocks_for(p, n_tokens);
+  if (!r) {
+    if (p->n_reqs == p->cap_reqs) {
+      int64_t nc = p->cap_reqs ? p->cap_reqs * 2 : 16;
+      orc_req *nr = (orc_req *)realloc(p->reqs, sizeof(orc_req) * (size_t)nc);
+      if (!nr) { free(prefix); return ORC_ERR_NOMEM; }
+      p->reqs = nr; p->cap_reqs = nc;
+    }
+    r = &p->reqs[p->n_reqs++];
+    memset(r, 0, sizeof(*r));
+    r->id = id;
+  }
+  r->state = ORC_ACTIVE;
+  r->n_tokens = n_tokens;
+  r->nb = nb;
+  r->n_shared = n_shared;
+  r->image_bytes = (uint64_t)(n_tokens - (int64_t)n_shared * p->BS) * p->bpt;
+  r->blocks = (int32_t *)malloc(sizeof(int32_t) * (size_t)(nb ? nb : 1));
+  if (n_shared) memcpy(r->blocks, prefix, sizeof(int32_t) * (size_t)n_shared);
+  free(prefix);
+  freeq_pop(p, nb - n_shared, r->blocks + n_shared);
+  ref_blocks(p, r->blocks, nb);
   if (out_blocks) memcpy(out_blocks, r->blocks, sizeof(int32_t) * (size_t)nb);
   return ORC_OK;
 }
@@ -309,8 +392,10 @@ int32_t orc_request_admit_into(orc_pool *p, uint64_t id, int64_t n_tokens, const
   r->n_tokens = n_tokens;
   r->nb = nb;
   r->image_bytes = (uint64_t)n_tokens * p->bpt;
+  r->n_shared = 0;
   r->blocks = (int32_t *)malloc(sizeof(int32_t) * (size_t)(nb ? nb : 1));
   memcpy(r->blocks, blocks, sizeof(int32_t) * (size_t)nb);
+  ref_blocks(p, r->blocks, nb);
   return ORC_OK;
 }
 
@@ -319,7 +404,7 @@ int32_t orc_request_release(orc_pool *p, uint64_t id) {
   orc_req *r = find_req(p, id);
   if (!r) return ORC_ERR_UNKNOWN_REQUEST;
   if (r->state == ORC_ACTIVE || r->state == ORC_RETAINED) drop_blocks(p, r);
-  if (r->state == ORC_HOST) drop_host_copy(p, r);
+  if (r->state == ORC_HOST) { drop_host_copy(p, r); drop_blocks(p, r); }   /* the copy, and the prefix it still refers to */
   int64_t i = r - p->reqs;
   memmove(p->reqs + i, p->reqs + i + 1, sizeof(orc_req) * (size_t)(p->n_reqs - i - 1));
   p->n_reqs -= 1;
@@ -345,10 +430,14 @@ static int32_t suspend_one(orc_pool *p, uint64_t id) {
   if (p->with_data) {
     r->image = (uint8_t *)malloc((size_t)(r->image_bytes ? r->image_bytes : 1));
     if (!r->image) { if (len) arena_remove(p, id); return ORC_ERR_NOMEM; }
-    orc_gather(p->data, r->image, p->L, p->H, p->D, p->e, p->BS, p->NB, r->blocks, r->n_tokens, p->layout);
+    /* only the private suffix is per-request state: the image is the gather over the private part of the table */
+    orc_gather(p->data, r->image, p->L, p->H, p->D, p->e, p->BS, p->NB, r->blocks + r->n_shared,
+               private_tokens(p, r), p->layout);
   }
   r->arena_off = off; r->arena_len = len;
-  drop_blocks(p, r);                 /* ids go to the free tail in logical order */
+  /* private blocks are let go in logical order (free tail when the last reference goes); the request keeps
+   * referring to its shared prefix, which therefore stays resident while the request waits on the host */
+  unref_blocks(p, r->blocks, r->n_shared, r->nb);
   r->state = ORC_HOST;               /* state 2 of Eq. 1 */
   p->st.suspends++; p->st.bytes_suspended += r->image_bytes;
   return ORC_OK;
@@ -360,6 +449,7 @@ static int32_t expire_one(orc_pool *p, uint64_t id) {
   if (r->state == ORC_HOST) {
     p->st.bytes_expired_from_host += r->image_bytes;
     drop_host_copy(p, r);
+    drop_blocks(p, r);               /* the shared prefix it still referred to */
   } else if (r->state == ORC_ACTIVE || r->state == ORC_RETAINED) {
     drop_blocks(p, r);
   } else {
@@ -370,11 +460,19 @@ static int32_t expire_one(orc_pool *p, uint64_t id) {
   return ORC_OK;
 }
 
-static int32_t resume_with_blocks(orc_pool *p, orc_req *r, int32_t *blocks) {
+/* `fresh` holds the nb - n_shared ids just taken for the private part (ownership passes to this function) */
+static int32_t resume_with_blocks(orc_pool *p, orc_req *r, int32_t *fresh) {
+  int32_t n_priv = r->nb - r->n_shared;
   if (p->with_data)
-    orc_scatter(p->data, r->image, p->L, p->H, p->D, p->e, p->BS, p->NB, blocks, r->n_tokens, p->layout);
+    orc_scatter(p->data, r->image, p->L, p->H, p->D, p->e, p->BS, p->NB, fresh, private_tokens(p, r), p->layout);
   drop_host_copy(p, r);
-  r->blocks = blocks;
+  ref_blocks(p, fresh, n_priv);
+  /* the table is the prefix the request never let go of, followed by the new private blocks */
+  int32_t *table = (int32_t *)malloc(sizeof(int32_t) * (size_t)(r->nb ? r->nb : 1));
+  if (r->n_shared) memcpy(table, r->blocks, sizeof(int32_t) * (size_t)r->n_shared);
+  if (n_priv) memcpy(table + r->n_shared, fresh, sizeof(int32_t) * (size_t)n_priv);
+  free(fresh); free(r->blocks);
+  r->blocks = table;
   r->state = ORC_ACTIVE;
   p->st.resumes++; p->st.bytes_resumed += r->image_bytes;
   return ORC_OK;
@@ -386,10 +484,11 @@ static int32_t resume_one(orc_pool *p, uint64_t id) {
   if (r->state == ORC_RETAINED) { r->state = ORC_ACTIVE; p->st.resident_resumes++; return ORC_RESIDENT; }
   if (r->state == ORC_EXPIRED) return ORC_RECOMPUTE;
   if (r->state != ORC_HOST) return ORC_ERR_BAD_STATE;
-  if ((int64_t)r->nb > p->n_free) { p->st.hbm_full_rejects++; return ORC_HBM_FULL; }
-  int32_t *blocks = (int32_t *)malloc(sizeof(int32_t) * (size_t)(r->nb ? r->nb : 1));
+  int32_t n_priv = r->nb - r->n_shared;
+  if ((int64_t)n_priv > p->n_free) { p->st.hbm_full_rejects++; return ORC_HBM_FULL; }
+  int32_t *blocks = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_priv ? n_priv : 1));
   if (!blocks) return ORC_ERR_NOMEM;
-  freeq_pop(p, r->nb, blocks);
+  freeq_pop(p, n_priv, blocks);
   return resume_with_blocks(p, r, blocks);
 }
 
@@ -398,7 +497,7 @@ int32_t orc_resume_from_host_into(orc_pool *p, uint64_t id, const int32_t *block
   orc_req *r = find_req(p, id);
   if (!r) return ORC_ERR_UNKNOWN_REQUEST;
   if (r->state != ORC_HOST) return ORC_ERR_BAD_STATE;
-  if (nb != r->nb) return ORC_ERR_INVALID_ARG;
+  if (nb != r->nb - r->n_shared) return ORC_ERR_INVALID_ARG;      /* the private part is what moves */
   /* every named block must be free, and named once */
   for (int32_t i = 0; i < nb; ++i) {
     int found = 0;
@@ -466,10 +565,22 @@ int32_t orc_pool_stats(orc_pool *p, orc_stats *out) {
   s.n_active = s.n_retained = s.n_host = s.n_expired = 0;
   for (int64_t i = 0; i < p->n_reqs; ++i) {
     const orc_req *r = &p->reqs[i];
-    if (r->state == ORC_ACTIVE) { s.n_active++; s.blocks_active += r->nb; }
-    if (r->state == ORC_RETAINED) { s.n_retained++; s.blocks_pinned += r->nb; }
+    if (r->state == ORC_ACTIVE) s.n_active++;
+    if (r->state == ORC_RETAINED) s.n_retained++;
     if (r->state == ORC_HOST) s.n_host++;
     if (r->state == ORC_EXPIRED) s.n_expired++;
+  }
+  /* a block is pinned when a suspended context (RETAINED, or on the host and still referring to its shared prefix)
+   * names it; every other held block is active.  Counted per distinct block, by scanning every table. */
+  for (int32_t b = 0; b < p->NB; ++b) {
+    int held = 0, pinned = 0;
+    for (int64_t i = 0; i < p->n_reqs; ++i) {
+      const orc_req *r = &p->reqs[i];
+      int32_t cnt = (r->state == ORC_ACTIVE || r->state == ORC_RETAINED) ? r->nb : (r->state == ORC_HOST ? r->n_shared : 0);
+      for (int32_t k = 0; k < cnt; ++k)
+        if (r->blocks[k] == b) { held = 1; if (r->state != ORC_ACTIVE) pinned = 1; }
+    }
+    if (pinned) s.blocks_pinned++; else if (held) s.blocks_active++;
   }
   s.host_capacity = p->host_capacity; s.host_used = 0; s.host_largest_hole = 0;
   uint64_t cursor = 0;
@@ -490,4 +601,24 @@ int64_t orc_free_queue(orc_pool *p, int32_t *out, int64_t cap) {
   if (!p) return -1;
   if (out) memcpy(out, p->freeq, sizeof(int32_t) * (size_t)(p->n_free < cap ? p->n_free : cap));
   return p->n_free;
+}
+
+/* the shared prefix a request refers to (any state but EXPIRED): its length in blocks, and the ids */
+int32_t orc_request_sharing(orc_pool *p, uint64_t id, int32_t *n_shared, int32_t *blocks, int32_t cap) {
+  if (!p) return ORC_ERR_INVALID_ARG;
+  orc_req *r = find_req(p, id);
+  if (!r) return ORC_ERR_UNKNOWN_REQUEST;
+  int32_t ns = (r->state == ORC_EXPIRED) ? 0 : r->n_shared;
+  if (n_shared) *n_shared = ns;
+  if (blocks) {
+    if (cap < ns) return ORC_ERR_INVALID_ARG;
+    if (ns) memcpy(blocks, r->blocks, sizeof(int32_t) * (size_t)ns);
+  }
+  return ORC_OK;
+}
+
+/* number of references to one block (0 = free), -1 for an id out of range */
+int32_t orc_block_refcount(orc_pool *p, int32_t blk) {
+  if (!p || blk < 0 || blk >= p->NB) return -1;
+  return p->refcnt[blk];
 }

@@ -27,7 +27,9 @@
  * Pins (tests, CPU only): the paper's worked byte counts, numpy fancy-indexing
  * on identity tables, a dictionary-based brute force on pools of <= 6 blocks,
  * round-trip identity under arbitrary relabelling, occupancy arithmetic of
- * Appendix A (42,548-block pool, 525-block contexts, 81 fit).
+ * Appendix A (42,548-block pool, 525-block contexts, 81 fit); for shared prefixes the
+ * paper's 5.4K + 3.0K token split (image = 983,040,000 bytes), conservation with
+ * reference counts, and brute force over two requests sharing a prefix.
  * Throughput of this code is a reported baseline only: parity unpinned.
  */
 #ifndef KVR_ORACLE_H
@@ -86,6 +88,15 @@ uint64_t orc_pool_bytes(orc_pool *);
 
 int32_t orc_request_admit(orc_pool *, uint64_t id, int64_t n_tokens, int32_t *out_blocks, int32_t cap);
 int32_t orc_request_admit_into(orc_pool *, uint64_t id, int64_t n_tokens, const int32_t *blocks, int32_t nb);
+/* Shared prefix (Section 2: the system prefix is shared through prefix caching and only the private suffix is
+ * per-request state).  The new request's first n_shared blocks are the donor's first n_shared blocks, reference
+ * counted; a block returns to the free queue when its last reference goes.  While such a request is on the host it
+ * keeps its references to the prefix (the prefix stays resident) and its image holds the private suffix only:
+ * tokens [n_shared*BS, n_tokens), (n_tokens - n_shared*BS) * bytes_per_token bytes. */
+int32_t orc_request_admit_sharing(orc_pool *, uint64_t id, int64_t n_tokens, uint64_t donor_id, int32_t n_shared,
+                                  int32_t *out_blocks, int32_t cap);
+int32_t orc_request_sharing(orc_pool *, uint64_t id, int32_t *n_shared, int32_t *blocks, int32_t cap);
+int32_t orc_block_refcount(orc_pool *, int32_t blk);
 int32_t orc_request_release(orc_pool *, uint64_t id);
 int32_t orc_retain_in_hbm(orc_pool *, const uint64_t *ids, int32_t n, int32_t *per_req);
 int32_t orc_suspend_to_host(orc_pool *, const uint64_t *ids, int32_t n, int32_t *per_req);

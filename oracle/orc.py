@@ -72,6 +72,12 @@ def lib():
         L.orc_request_admit_into.argtypes = [vp, u64, i64, pi32, i32]
         L.orc_request_release.restype = i32
         L.orc_request_release.argtypes = [vp, u64]
+        L.orc_request_admit_sharing.restype = i32
+        L.orc_request_admit_sharing.argtypes = [vp, u64, i64, u64, i32, pi32, i32]
+        L.orc_request_sharing.restype = i32
+        L.orc_request_sharing.argtypes = [vp, u64, pi32, pi32, i32]
+        L.orc_block_refcount.restype = i32
+        L.orc_block_refcount.argtypes = [vp, i32]
         for name in ("orc_retain_in_hbm", "orc_suspend_to_host", "orc_expire", "orc_resume_from_host"):
             f = getattr(L, name)
             f.restype = i32
@@ -167,6 +173,25 @@ class OrcPool:
 
     def release(self, rid):
         return lib().orc_request_release(self._h, rid)
+
+    def admit_sharing(self, rid, n_tokens, donor, n_shared):
+        nb = (n_tokens + self.geom[4] - 1) // self.geom[4] if n_tokens >= 0 else 0
+        out = np.zeros(max(nb, 1), dtype=np.int32)
+        st = lib().orc_request_admit_sharing(self._h, rid, n_tokens, donor, n_shared, _i32p(out), nb)
+        return st, (out[:nb].copy() if st == OK else None)
+
+    def sharing(self, rid):
+        """(status, shared-prefix block ids the request refers to)."""
+        ns = C.c_int32()
+        st = lib().orc_request_sharing(self._h, rid, C.byref(ns), None, 0)
+        if st != OK:
+            return st, None
+        out = np.zeros(max(ns.value, 1), dtype=np.int32)
+        lib().orc_request_sharing(self._h, rid, None, _i32p(out), ns.value)
+        return st, out[:ns.value].copy()
+
+    def refcount(self, blk):
+        return int(lib().orc_block_refcount(self._h, blk))
 
     def _batch(self, fn, ids):
         ids = np.ascontiguousarray(ids, dtype=np.uint64)
