@@ -8,7 +8,7 @@ image and re-admit it, resume the batch (block allocation, host-to-device copies
 kernel).  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                  [--workload llama3_8b|tiny|gqa64|trace|longctx|paper_70b_tp4]
+                  [--workload llama3_8b|tiny|gqa64|trace|longctx|paper_70b_tp4|paper_shape]
                   [--route staged|mapped|dma2d] [--kernel warp|bulk] [--layout layer|block] [--arena host|device]
 """
 import argparse
@@ -37,6 +37,21 @@ def peaks():
     if os.path.exists(path):
         return json.load(open(path))["hbm_gbs"], "measured"
     return 6650.0, "fallback"
+
+
+def l2_residues():
+    """Bytes a mover launch has written but not yet evicted to DRAM when it ends (ncu capture on a small case:
+    DRAM reads equal the payload, DRAM writes fall short of it by this constant), per kernel and direction; the
+    summary under profiles/ carries them on one 'l2_residue_bytes' line."""
+    path = os.path.join(ROOT, "profiles", "ncu_dram_traffic_movers.md")
+    out = {}
+    if os.path.exists(path):
+        for line in open(path):
+            if line.startswith("l2_residue_bytes "):
+                for kv in line.split()[1:]:
+                    k, v = kv.split("=")
+                    out[k] = float(v)
+    return out, "profiles/ncu_dram_traffic_movers.md"
 
 
 class ClockSampler:
@@ -96,6 +111,22 @@ def build_workload(name, n_requests_cap=None, overrides=None):
     used = int(sum(-(-int(n) // bs) for n in lens))
     fillers = occupancy_fillers(w.num_blocks, bs, used, w.occupancy, seed) if w.occupancy else np.zeros(0, np.int64)
     return w, seed, lens, fillers
+
+
+def engine_kwargs(args, kvr):
+    """Engine settings from the command line; 0 / unset leaves the library's own default in place."""
+    kw = dict(chunk_bytes=args.chunk_mib << 20, staging_slots=args.slots, max_ctas=args.max_ctas,
+              kernel={"warp": kvr.KERNEL_WARP, "bulk": kvr.KERNEL_BULK}[args.kernel],
+              ramp_start_bytes=args.ramp_mib << 20, copy_piece_bytes=args.copy_piece_mib << 20)
+    if args.bulk_shape:
+        kw["bulk_shape"] = tuple(int(x) for x in args.bulk_shape.split(","))
+    return kw
+
+
+def staging_note(args):
+    slot, n = (args.chunk_mib or 64), (args.slots or 16)
+    return {"slot_mib": slot, "slots_per_direction": n, "staging_mib_total": 2 * slot * n,
+            "largest_launch_mib": slot * (n - 1), "library_default": not (args.chunk_mib or args.slots)}
 
 
 def cpu_oracle_sample(geom, tokens, threads=1):
@@ -244,9 +275,7 @@ def run_longctx(args):
     sink = torch.zeros(1024, dtype=torch.int64, device="cuda")
     torch.cuda.synchronize()
     pool = kvr.Pool(*w.geom, NB, host_cap, initial_free_order=free_order(seed, NB), device=local,
-                    device_pool=dev_pool.data_ptr(), chunk_bytes=args.chunk_mib << 20, staging_slots=args.slots,
-                    kernel={"warp": kvr.KERNEL_WARP, "bulk": kvr.KERNEL_BULK}[args.kernel], max_ctas=args.max_ctas,
-                    flags=kvr.PROFILE)
+                    device_pool=dev_pool.data_ptr(), flags=kvr.PROFILE, **engine_kwargs(args, kvr))
     link = link_peak(torch, pool, host_cap)            # while the arena is still empty
     ids = list(range(n_req))
     for rid in ids:
@@ -310,7 +339,7 @@ def run_longctx(args):
         "config": {"workload": "longctx", "geometry": dict(zip(("layers", "kv_heads", "head_dim", "dtype_bytes", "block_size"), w.geom)),
                    "requests_requested": w.n_requests, "requests_run": n_req, "tokens_per_request": n_tok,
                    "bytes_per_direction": half_bytes, "num_blocks": NB, "load_buffer_bytes": load_bytes,
-                   "kernel": args.kernel, "chunk_mib": args.chunk_mib, "max_ctas": args.max_ctas},
+                   "kernel": args.kernel, "staging": staging_note(args), "max_ctas": args.max_ctas},
         "interference": {
             "alone_one_direction_at_a_time": seq, "overlapped": ovl, "overlapped_with_load": ovl_load,
             "load_alone_gbs": load_alone, "load_alone_frac_of_hbm_peak": load_alone / peak,
@@ -323,6 +352,9 @@ def run_longctx(args):
         "roofline": {"bound": "hbm", "peak": peak, "unit": "GB/s", "tile_bytes": BS * H * D * e,
                      "gather_frac": 2 * st["gather_bytes"] / max(st["gather_ms"], 1e-9) / 1e6 / peak,
                      "scatter_frac": 2 * st["scatter_bytes"] / max(st["scatter_ms"], 1e-9) / 1e6 / peak,
+                     "gather_launches": int(st["gather_launches"]), "scatter_launches": int(st["scatter_launches"]),
+                     "mover_busy_us_per_gb": {"gather": 1e3 * st["gather_ms"] / max(st["gather_bytes"] / 1e9, 1e-9),
+                                              "scatter": 1e3 * st["scatter_ms"] / max(st["scatter_bytes"] / 1e9, 1e-9)},
                      "note": "CUDA events around every mover launch, all phases of this run"},
         "gpu_launches": int(st["gather_launches"] + st["scatter_launches"]),
     }
@@ -359,8 +391,7 @@ def run_trace(args):
         view[i:i + (1 << 28)].normal_(generator=gen)
     torch.cuda.synchronize()
     pool = kvr.Pool(*w.geom, w.num_blocks, host_cap, initial_free_order=free_order(seed, w.num_blocks), device=local,
-                    device_pool=dev_pool.data_ptr(), chunk_bytes=args.chunk_mib << 20, staging_slots=args.slots,
-                    kernel={"warp": kvr.KERNEL_WARP, "bulk": kvr.KERNEL_BULK}[args.kernel], flags=kvr.PROFILE)
+                    device_pool=dev_pool.data_ptr(), flags=kvr.PROFILE, **engine_kwargs(args, kvr))
     link = link_peak(torch, pool, host_cap)
     prices = (0.0176, 0.02, 1.91)                           # the paper's H100 NVL price vector, as context constants
     mean_img = float(np.mean(lengths)) * bpt
@@ -402,18 +433,48 @@ def run_trace(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": "trace", "requests": int(w.n_requests), "num_blocks": w.num_blocks, "host_capacity": host_cap,
                    "lambda_per_s": lam, "w_ref_s": w_ref, "hbm_grace_s": 60.0, "t2_s": cs["t2"], "branch": "cpu_ttl",
-                   "admission": "replay", "kernel": args.kernel, "chunk_mib": args.chunk_mib},
+                   "admission": "replay", "kernel": args.kernel, "staging": staging_note(args)},
         "trace": {"bytes_suspended": st["bytes_suspended"], "bytes_resumed": st["bytes_resumed"],
                   "bytes_expired_from_host": st["bytes_expired_from_host"], "controller": cs,
                   "outcomes": {"%s:%d" % k: v for k, v in sorted(outcomes.items())},
                   "gpu_cost_per_request": cs["gpu_cost"] / w.n_requests},
         "roofline": {"bound": "hbm", "peak": peak, "unit": "GB/s", "gather_frac": g_gbs / peak, "scatter_frac": s_gbs / peak,
+                     "gather_launches": int(st["gather_launches"]), "scatter_launches": int(st["scatter_launches"]),
+                     "mover_busy_us_per_gb": {"gather": 1e3 * st["gather_ms"] / max(st["gather_bytes"] / 1e9, 1e-9),
+                                              "scatter": 1e3 * st["scatter_ms"] / max(st["scatter_bytes"] / 1e9, 1e-9)},
                      "note": "per-request moves of ~0.6 GiB: launches are smaller than in the batched configurations"},
         "host_link": link, "clocks": clocks, "gpu_launches": int(st["gather_launches"] + st["scatter_launches"]),
     }
     print(json.dumps(out))
     ctl.close()
     pool.close()
+
+
+def probe_links(group, pool, host_cap, payload, torch):
+    """Every rank measures its own link over its own arena: once alone (ranks take turns between barriers) and once
+    with all ranks copying at the same time, which shows what sharing the host's DRAM and root ports costs."""
+    alone = None
+    for r in range(group.world):
+        group.barrier()
+        if group.rank == r:
+            alone = link_peak(torch, pool, host_cap, payload=payload if group.world == 1 else 0)
+    group.barrier()
+    together = None
+    if group.world > 1:
+        n = min(host_cap // 4096 * 4096, 2 << 30)
+        st, d2h, h2d = pool.probe_link(n, 6)
+        together = (d2h, h2d) if st == 0 else (0.0, 0.0)
+        group.barrier()
+    # everybody learns everybody's figures: a vector with this rank's slots filled, summed over ranks
+    vec = [0.0] * (5 * group.world)
+    vec[5 * group.rank:5 * group.rank + 5] = [alone["d2h_best_gbs"], alone["h2d_best_gbs"],
+                                              together[0] if together else 0.0, together[1] if together else 0.0,
+                                              float(pool.numa_node)]
+    allv = group.sum(vec)
+    per_rank = [{"rank": r, "d2h_alone_gbs": allv[5 * r], "h2d_alone_gbs": allv[5 * r + 1],
+                 "d2h_all_ranks_at_once_gbs": allv[5 * r + 2] or None, "h2d_all_ranks_at_once_gbs": allv[5 * r + 3] or None,
+                 "arena_numa_node": int(allv[5 * r + 4])} for r in range(group.world)]
+    return alone, per_rank
 
 
 def run_ours(args):
@@ -423,10 +484,12 @@ def run_ours(args):
     from paper_2608_30830_b200.multi import Group, env_ranks, fit_requests
 
     rank, world, local = env_ranks()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
-    torch.cuda.set_device(local)
-    group = Group("nccl", torch.device("cuda", local))
+    dry = args.dry_run
+    if not dry:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+        torch.cuda.set_device(local)
+    group = Group("gloo" if dry else "nccl", None if dry else torch.device("cuda", local))
 
     # every rank runs its own replica of the workload (own pool, own host link, own arena): weak scaling.
     # Scale rule: the arenas of all ranks come out of the same host DRAM; keep geometry and lengths and
@@ -434,77 +497,98 @@ def run_ours(args):
     ov = {"num_blocks": args.num_blocks, "requests": args.requests, "fixed_tokens": args.fixed_tokens}
     w, seed, lens, fillers = build_workload(args.workload, None, ov)
     bpt = kvr.bytes_per_token(*w.geom[:4])
+    L, H, D, e, BS = w.geom
+    shared_blocks = 0 if args.no_share else int(w.extra.get("shared_tokens", 0)) // BS
+    shared_tokens = shared_blocks * BS
     requested = len(lens)
     avail = int(open("/proc/meminfo").read().split("MemAvailable:")[1].split()[0]) * 1024
-    keep = int(group.max([-fit_requests(lens, bpt, avail, world)])[0]) * -1      # the same count on every rank
+    keep = int(group.max([-fit_requests(lens - shared_tokens, bpt, avail, world)])[0]) * -1      # the same count on every rank
     if keep != requested:
         w, seed, lens, fillers = build_workload(args.workload, keep, ov)
-    L, H, D, e, BS = w.geom
-    payload = int(lens.sum()) * bpt
+    if shared_blocks:
+        # the fillers were sized as if every request owned its prefix: recompute them for the shared layout
+        used = shared_blocks + int(sum(-(-int(n) // BS) - shared_blocks for n in lens))
+        fillers = occupancy_fillers(w.num_blocks, BS, used, w.occupancy, seed) if w.occupancy else fillers
+    payload = int((lens - shared_tokens).sum()) * bpt
     lone_tokens = 8192
     small_k = int(np.argmin(fillers)) if len(fillers) else None     # request used for the retain / expire rows
     small_tokens = int(fillers[small_k]) if small_k is not None else 0
-    host_cap = -(-(payload + len(lens) * 4096 + (lone_tokens + small_tokens) * bpt + (64 << 20)) // 4096) * 4096
+    unshared_extra = int(lens.sum()) * bpt if shared_blocks else 0   # the comparison pass without sharing needs room too
+    host_cap = -(-(max(payload, unshared_extra) + len(lens) * 4096 + (lone_tokens + small_tokens) * bpt + (64 << 20)) // 4096) * 4096
 
-    # pool bytes: bf16 N(0,1) drawn on the device from a seeded generator
-    pool_bytes = w.num_blocks * BS * bpt
-    dev_pool = torch.empty(pool_bytes, dtype=torch.uint8, device="cuda")
-    gen = torch.Generator(device="cuda")
-    gen.manual_seed(seed + rank)
-    view = dev_pool.view(torch.bfloat16)
-    step_elems = 1 << 28
-    for i in range(0, view.numel(), step_elems):
-        view[i:i + step_elems].normal_(generator=gen)
-    torch.cuda.synchronize()
-
-    route = {"staged": kvr.ROUTE_STAGED, "mapped": kvr.ROUTE_MAPPED, "dma2d": kvr.ROUTE_DMA2D}[args.route]
+    route = {"auto": kvr.ROUTE_AUTO, "staged": kvr.ROUTE_STAGED, "mapped": kvr.ROUTE_MAPPED, "dma2d": kvr.ROUTE_DMA2D}[args.route]
     layout = {"layer": kvr.LAYER_MAJOR, "block": kvr.BLOCK_MAJOR}[args.layout]
-    kernel = {"warp": kvr.KERNEL_WARP, "bulk": kvr.KERNEL_BULK}[args.kernel]
-    dev_arena = torch.empty(host_cap, dtype=torch.uint8, device="cuda") if args.arena == "device" else None
-    pool = kvr.Pool(*w.geom, w.num_blocks, host_cap, initial_free_order=free_order(seed, w.num_blocks),
-                    device=local, device_pool=dev_pool.data_ptr(), route=route, kernel=kernel,
-                    host_arena=dev_arena.data_ptr() if dev_arena is not None else None,
-                    chunk_bytes=args.chunk_mib << 20, staging_slots=args.slots, max_ctas=args.max_ctas,
-                    flags=kvr.PROFILE, layout=layout)
+    dev_pool = dev_arena = None
+    if dry:
+        pool = kvr.Pool(*w.geom, w.num_blocks, host_cap, initial_free_order=free_order(seed, w.num_blocks),
+                        flags=kvr.METADATA_ONLY, layout=layout)
+    else:
+        # pool bytes: bf16 N(0,1) drawn on the device from a seeded generator
+        pool_bytes = w.num_blocks * BS * bpt
+        dev_pool = torch.empty(pool_bytes, dtype=torch.uint8, device="cuda")
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(seed + rank)
+        view = dev_pool.view(torch.bfloat16)
+        step_elems = 1 << 28
+        for i in range(0, view.numel(), step_elems):
+            view[i:i + step_elems].normal_(generator=gen)
+        torch.cuda.synchronize()
+        dev_arena = torch.empty(host_cap, dtype=torch.uint8, device="cuda") if args.arena == "device" else None
+        pool = kvr.Pool(*w.geom, w.num_blocks, host_cap, initial_free_order=free_order(seed, w.num_blocks),
+                        device=local, device_pool=dev_pool.data_ptr(), route=route,
+                        host_arena=dev_arena.data_ptr() if dev_arena is not None else None,
+                        flags=kvr.PROFILE, layout=layout, **engine_kwargs(args, kvr))
+
+    # the link peaks, before anything lives in the arena: per rank, alone and all at once
+    link, per_rank_links = (None, None)
+    if not dry and dev_arena is None:
+        link, per_rank_links = probe_links(group, pool, host_cap, payload, torch)
 
     # live set: the batch and the fillers, admitted in a seeded interleaved order (fragmented placement)
     ids = list(range(len(lens)))
     filler_ids = list(range(1000, 1000 + len(fillers)))
+    PREFIX = 900
+    if shared_blocks:
+        assert pool.admit(PREFIX, shared_tokens)[0] == kvr.OK          # the system prefix, computed once
     order = [(i, int(n)) for i, n in zip(ids, lens)] + [(i, int(n)) for i, n in zip(filler_ids, fillers)]
     np.random.default_rng(seed).shuffle(order)
     for rid, n in order:
-        st, _ = pool.admit(rid, n)
+        if shared_blocks and rid < 900:
+            st, _ = pool.admit_sharing(rid, n, PREFIX, shared_blocks)
+        else:
+            st, _ = pool.admit(rid, n)
         assert st == kvr.OK, (rid, n, st, kvr.last_error())
+    if shared_blocks:
+        assert pool.release(PREFIX) == kvr.OK                          # its blocks live on through the sharers' references
     occupancy = 1.0 - pool.stats()["blocks_free"] / w.num_blocks
     small = filler_ids[small_k] if small_k is not None else None
 
-    link = link_peak(torch, pool, host_cap, payload=payload) if (rank == 0 and dev_arena is None) else None
-
     def barrier():
-        torch.cuda.synchronize()
+        if not dry:
+            torch.cuda.synchronize()
         group.barrier()
 
     last_resume_ms = []
 
-    def one_step():
+    def one_step(batch=ids, low_latency=args.low_latency):
         """Returns (device_ms_suspend, device_ms_resume, wall_s)."""
         t0 = time.perf_counter()
         if small is not None:                          # HBM retention: nothing moves, resume is resident
             assert pool.retain_in_hbm([small])[0] == kvr.OK
             assert pool.resume_from_host([small])[0] == kvr.RESIDENT
-        st, per = pool.suspend_to_host(ids)
+        st, per = pool.suspend_to_host(batch)
         assert st == kvr.OK, (st, per, kvr.last_error())
         assert pool.wait() == kvr.OK, kvr.last_error()
-        sus = max(pool.latency(r)[2] for r in ids)
+        sus = 0.0 if dry else max(pool.latency(r)[2] for r in batch)
         if small is not None:                          # host copy expires, resume answers recompute, re-admit
             assert pool.suspend_to_host([small], kvr.SYNC)[0] == kvr.OK
             assert pool.expire([small])[0] == kvr.OK
             assert pool.resume_from_host([small])[0] == kvr.RECOMPUTE
             assert pool.admit(small, small_tokens)[0] == kvr.OK
-        st, per = pool.resume_from_host(ids, kvr.LOW_LATENCY if args.low_latency else 0)
+        st, per = pool.resume_from_host(batch, kvr.LOW_LATENCY if low_latency else 0)
         assert st == kvr.OK, (st, per, kvr.last_error())
         assert pool.wait() == kvr.OK, kvr.last_error()
-        per_req = [pool.latency(r)[2] for r in ids]
+        per_req = [0.0 if dry else pool.latency(r)[2] for r in batch]
         last_resume_ms[:] = per_req
         res = max(per_req)
         return sus, res, time.perf_counter() - t0
@@ -514,12 +598,13 @@ def run_ours(args):
     sampler = ClockSampler(local)
     s0 = pool.stats()
     barrier()
-    sampler.start()
+    if not dry:
+        sampler.start()
     t_begin = time.perf_counter()
     steps = [one_step() for _ in range(args.steps)]
     barrier()
     wall = time.perf_counter() - t_begin
-    clocks = sampler.stop()
+    clocks = sampler.stop() if not dry else None
     s1 = pool.stats()
 
     sus_ms = float(np.sum([s[0] for s in steps]))
@@ -529,10 +614,22 @@ def run_ours(args):
     payload_all = group.sum([payload])[0]
     K = args.steps
     moved = 2.0 * payload_all * K                      # bytes suspended + bytes resumed, all ranks
-    value = moved / dev_s / 1e9
+    value = moved / dev_s / 1e9 if dev_s > 0 else None
     e2e = moved / wall / 1e9
 
-    if rank == 0:
+    if rank == 0 and dry:
+        d = {k: s1[k] - s0[k] for k in ("suspends", "resumes", "bytes_suspended", "bytes_resumed")}
+        print(json.dumps({
+            "metric": METRIC, "value": None, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "ms_per_step": 1e3 * wall / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "u8", "data": "synthetic", "dry_run": True,
+            "config": {"workload": w.name, "requests_requested": requested, "requests_run": len(ids),
+                       "note": "launcher and bookkeeping check without a GPU: metadata-only pools, gloo ranks, nothing moved"},
+            "bookkeeping": {"bytes_suspended_per_step_all_ranks": payload_all,
+                            "bytes_suspended_this_rank": int(d["bytes_suspended"]), "suspends_this_rank": int(d["suspends"])},
+            "gpu_launches": 0}))
+
+    if rank == 0 and not dry:
         # kernels inside the timed region (profiling events around every launch)
         d = {k: s1[k] - s0[k] for k in ("gather_launches", "scatter_launches", "gather_bytes", "scatter_bytes",
                                         "gather_ms", "scatter_ms", "gather_kernel_ms", "scatter_kernel_ms", "d2h_bytes", "h2d_bytes", "desc_bytes",
@@ -540,34 +637,46 @@ def run_ours(args):
         peak, peak_kind = peaks()
         g_gbs = 2 * d["gather_bytes"] / max(d["gather_ms"], 1e-9) / 1e6
         s_gbs = 2 * d["scatter_bytes"] / max(d["scatter_ms"], 1e-9) / 1e6
-        name, ach = ("kvr::move_warp<gather>", g_gbs) if g_gbs <= s_gbs else ("kvr::move_warp<scatter>", s_gbs)
-        if args.kernel == "bulk":
-            name = name.replace("move_warp", "move_bulk")
-        # DRAM traffic per launch: ncu measured read+write = 0.979 x the algorithmic bytes on a 1 GiB chunk
-        # (ncu --set full capture of the gather on a small case); traffic grows in proportion to the bytes of a launch
-        launches = max(d["gather_launches"] if g_gbs <= s_gbs else d["scatter_launches"], 1)
-        alg_per_launch = 2 * (d["gather_bytes"] if g_gbs <= s_gbs else d["scatter_bytes"]) / launches
+        slower = "gather" if g_gbs <= s_gbs else "scatter"
+        name = "kvr::move_%s<%s>" % (args.kernel, slower)
+        ach = min(g_gbs, s_gbs)
+        # DRAM traffic per launch: ncu measured, for this kernel and direction on a small case, reads = payload and
+        # writes = payload minus a constant residue still in L2 at kernel end; reads and writes grow with the payload
+        residues, residue_file = l2_residues()
+        launches = max(d[slower + "_launches"], 1)
+        alg_per_launch = 2 * d[slower + "_bytes"] / launches
+        residue = residues.get("%s_%s" % (slower, args.kernel))
         same_run = None if args.no_extras else copy_peak_same_run(torch)
+
+        def side(gbs, key):
+            n = max(d[key + "_launches"], 1)
+            r = residues.get("%s_%s" % (key, args.kernel))
+            alg = 2 * d[key + "_bytes"] / n
+            return {"gbs": gbs, "frac": gbs / peak, "launches": d[key + "_launches"], "avg_us": 1e3 * d[key + "_ms"] / n,
+                    "avg_launch_mib": d[key + "_bytes"] / n / 2**20, "algorithmic_bytes_per_launch": alg,
+                    "traffic": None if r is None else max(alg - r, 0.0),
+                    "mover_busy_us_per_gb": 1e3 * d[key + "_ms"] / max(d[key + "_bytes"] / 1e9, 1e-9)}
         roofline = {"bound": "hbm", "kernel": name, "achieved": ach, "peak": peak, "unit": "GB/s",
                     "copy_peak_this_gpu_this_run": same_run,
                     "frac": ach / peak, "peak_source": peak_kind + " copy bandwidth, read+write bytes",
                     "algorithmic_bytes_per_launch": alg_per_launch,
-                    "traffic": 0.979 * alg_per_launch,
-                    "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum on a 1 GiB chunk, scaled by bytes per launch",
+                    "traffic": None if residue is None else max(alg_per_launch - residue, 0.0),
+                    "traffic_source": None if residue is None else
+                    "%s: ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel and direction on a small case "
+                    "(reads = payload, writes = payload - %.1f MB still in L2 at kernel end), applied to this run's "
+                    "bytes per launch" % (residue_file, residue / 1e6),
                     "in_kernel": {
                         "what": "the same launches timed by the kernels themselves: earliest CTA start to latest CTA end "
                                 "(%globaltimer), i.e. without the launch and completion latency the events include",
                         "gather_frac": 2 * d["gather_bytes"] / max(d["gather_kernel_ms"], 1e-9) / 1e6 / peak,
                         "scatter_frac": 2 * d["scatter_bytes"] / max(d["scatter_kernel_ms"], 1e-9) / 1e6 / peak},
-                    "gather": {"gbs": g_gbs, "frac": g_gbs / peak, "launches": d["gather_launches"],
-                               "avg_us": 1e3 * d["gather_ms"] / max(d["gather_launches"], 1)},
-                    "scatter": {"gbs": s_gbs, "frac": s_gbs / peak, "launches": d["scatter_launches"],
-                                "avg_us": 1e3 * d["scatter_ms"] / max(d["scatter_launches"], 1)}}
+                    "gather": side(g_gbs, "gather"), "scatter": side(s_gbs, "scatter")}
 
         # the kernels alone, at the size of the whole batch: HBM -> HBM
         alone = None
         free_b, _ = torch.cuda.mem_get_info()
-        need = payload + len(ids) * 256
+        whole = int(lens.sum()) * bpt
+        need = whole + len(ids) * 256
         if free_b > need + (2 << 30) and not args.no_extras:
             buf = torch.empty(need, dtype=torch.uint8, device="cuda")
             best = {}
@@ -577,8 +686,8 @@ def run_ours(args):
                     st, _ = fn(ids, buf.data_ptr(), need, kvr.SYNC)
                     assert st == kvr.OK, kvr.last_error()
                     ts.append(max(pool.latency(r)[2] for r in ids))
-                best[direction] = {"best_gbs": 2 * payload / min(ts[2:]) / 1e6,
-                                   "median_gbs": 2 * payload / float(np.median(ts[2:])) / 1e6}
+                best[direction] = {"best_gbs": 2 * whole / min(ts[2:]) / 1e6,
+                                   "median_gbs": 2 * whole / float(np.median(ts[2:])) / 1e6}
                 best[direction]["frac"] = best[direction]["median_gbs"] / peak
             alone = best
             del buf
@@ -602,6 +711,35 @@ def run_ours(args):
                     "timing": "host clock, call entry to return of the synchronous call"}
             pool.release(5000)
 
+        # shared prefix: what the same contexts cost when every request owns its whole context
+        sharing = None
+        if shared_blocks:
+            one = ids[0]
+            t0 = time.perf_counter()
+            assert pool.suspend_to_host([one], kvr.SYNC)[0] == kvr.OK
+            t1 = time.perf_counter()
+            assert pool.resume_from_host([one], kvr.SYNC)[0] == kvr.OK
+            t2 = time.perf_counter()
+            sharing = {"shared_tokens": shared_tokens, "context_tokens": int(lens[0]), "private_tokens": int(lens[0]) - shared_tokens,
+                       "bytes_per_suspend": (int(lens[0]) - shared_tokens) * bpt,
+                       "lone_suspend_ms": 1e3 * (t1 - t0), "lone_resume_ms": 1e3 * (t2 - t1),
+                       "batch_suspend_ms": sus_ms / K, "batch_resume_ms": res_ms / K}
+            if not args.no_extras:
+                for rid in ids:
+                    assert pool.release(rid) == kvr.OK
+                ok = all(pool.admit(rid, int(n))[0] == kvr.OK for rid, n in zip(ids, lens))
+                if ok:
+                    u = [one_step(ids, False) for _ in range(2)][-1]
+                    t0 = time.perf_counter()
+                    assert pool.suspend_to_host([one], kvr.SYNC)[0] == kvr.OK
+                    t1 = time.perf_counter()
+                    assert pool.resume_from_host([one], kvr.SYNC)[0] == kvr.OK
+                    t2 = time.perf_counter()
+                    sharing["without_sharing"] = {"bytes_per_suspend": int(lens[0]) * bpt, "lone_suspend_ms": 1e3 * (t1 - t0),
+                                                  "lone_resume_ms": 1e3 * (t2 - t1), "batch_suspend_ms": u[0], "batch_resume_ms": u[1]}
+                    sharing["bytes_ratio"] = int(lens[0]) / (int(lens[0]) - shared_tokens)
+                    sharing["lone_resume_speedup"] = sharing["without_sharing"]["lone_resume_ms"] / sharing["lone_resume_ms"]
+
         sus_gbs = payload_all * K / sus_ms / 1e6
         res_gbs = payload_all * K / res_ms / 1e6
         if link is None:        # device-memory tier: no host link on the path; the bound is HBM
@@ -609,8 +747,12 @@ def run_ours(args):
                          "suspend_frac_of_hbm_peak": 2 * sus_gbs / world / peak, "resume_frac_of_hbm_peak": 2 * res_gbs / world / peak}
         else:
             host_link = dict(link)
-            host_link.update({"suspend_gbs": sus_gbs, "suspend_frac_of_d2h_peak": sus_gbs / world / link["d2h_best_gbs"],
-                              "resume_gbs": res_gbs, "resume_frac_of_h2d_peak": res_gbs / world / link["h2d_best_gbs"]})
+            d2h_sum = sum(r["d2h_alone_gbs"] for r in per_rank_links)
+            h2d_sum = sum(r["h2d_alone_gbs"] for r in per_rank_links)
+            host_link.update({"suspend_gbs": sus_gbs, "suspend_frac_of_d2h_peak": sus_gbs / d2h_sum,
+                              "resume_gbs": res_gbs, "resume_frac_of_h2d_peak": res_gbs / h2d_sum,
+                              "per_rank": per_rank_links,
+                              "peak_note": "fractions are against the sum over ranks of each rank's own link measured alone"})
             if "d2h_sustained_gbs" in link:
                 host_link.update({"suspend_frac_of_d2h_sustained": sus_gbs / world / link["d2h_sustained_gbs"],
                                   "resume_frac_of_h2d_sustained": res_gbs / world / link["h2d_sustained_gbs"]})
@@ -623,9 +765,10 @@ def run_ours(args):
             "dtype": "u8", "data": "synthetic",
             "config": {"workload": w.name, "geometry": dict(zip(("layers", "kv_heads", "head_dim", "dtype_bytes", "block_size"), w.geom)),
                        "num_blocks": w.num_blocks, "requests_requested": requested, "requests_run": len(ids),
-                       "tokens": int(lens.sum()), "payload_bytes_per_direction": payload,
+                       "tokens": int(lens.sum()), "shared_prefix_tokens": shared_tokens, "payload_bytes_per_direction": payload,
                        "occupancy_before_suspend": occupancy, "route": args.route, "arena": args.arena, "layout": args.layout, "kernel": args.kernel,
-                       "chunk_mib": args.chunk_mib, "staging_slots": args.slots, "low_latency_resume": bool(args.low_latency), "seed": seed,
+                       "staging": staging_note(args), "low_latency_resume": bool(args.low_latency), "seed": seed,
+                       "arena_numa_node": pool.numa_node,
                        "l2": "inputs (tens of GiB) are far larger than L2; no flush needed",
                        "timing": "value: CUDA events, first enqueued work to last byte landed, summed over the two batched moves of each step; e2e: host clock around the K steps"},
             "e2e": {"value": e2e, "unit": "GB/s",
@@ -633,13 +776,13 @@ def run_ours(args):
                     "d2h_bytes_per_step": int(d["d2h_bytes"] / K)},
             "gpu_launches": int(d["gather_launches"] + d["scatter_launches"]),
             "clocks": clocks, "roofline": roofline, "kernels_alone": alone, "host_link": host_link,
-            "resume_latency_8k": lone,
+            "resume_latency_8k": lone, "sharing": sharing,
             "resume_latency_in_batch": {
                 "what": "device time from the batched resume's first enqueued work until each request's last byte landed "
                         "(requests complete in the order given); last timed step",
                 "first_ms": float(min(last_resume_ms)), "median_ms": float(np.median(last_resume_ms)),
                 "last_ms": float(max(last_resume_ms)),
-                "batch_ms_per_8k_tokens": float(max(last_resume_ms)) * 8192.0 / float(lens.sum())},
+                "batch_ms_per_8k_tokens": float(max(last_resume_ms)) * 8192.0 / float((lens - shared_tokens).sum())},
             "cpu_baseline": {"value": cpu["gbs"], "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample,
                              "suspend_s": cpu["suspend_s"], "resume_s": cpu["resume_s"],
                              "all_cores": None if args.no_extras else
@@ -650,6 +793,19 @@ def run_ours(args):
     group.close()
 
 
+def relaunch_under_torchrun(args):
+    """`python bench.py --gpus N` started plainly: start the N ranks (one per GPU) and pass their output through."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")               # the rank count must stay visible in the job's log
+    return subprocess.call(cmd, env=env)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -657,11 +813,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama3_8b", choices=list(CONFIGS))
-    ap.add_argument("--route", default="staged", choices=["staged", "mapped", "dma2d"])
+    ap.add_argument("--route", default="staged", choices=["auto", "staged", "mapped", "dma2d"])
     ap.add_argument("--layout", default="layer", choices=["layer", "block"], help="pool layout: layer-major or block-major")
     ap.add_argument("--kernel", default="bulk", choices=["warp", "bulk"])
-    ap.add_argument("--chunk-mib", type=int, default=1024, help="staging slot size; the library's own default is 512")
-    ap.add_argument("--slots", type=int, default=2)
+    ap.add_argument("--chunk-mib", type=int, default=0, help="staging slot size (0 = the library's default, 64)")
+    ap.add_argument("--slots", type=int, default=0, help="staging slots per direction (0 = the library's default, 16)")
+    ap.add_argument("--ramp-mib", type=int, default=0, help="size limit of a move's first chunk (0 = library default, 256)")
+    ap.add_argument("--copy-piece-mib", type=int, default=int(os.environ.get("KVR_COPY_PIECE_MIB", "0")),
+                    help="largest single link copy (0 = library default, 64)")
+    ap.add_argument("--bulk-shape", default=os.environ.get("KVR_BULK_SHAPE", ""), help="bulk mover shape: warps,stages,piece_bytes")
     ap.add_argument("--arena", default="host", choices=["host", "device"],
                     help="where the second tier lives: pinned host memory, or device memory (stand-in for a peer GPU)")
     ap.add_argument("--max-ctas", type=int, default=0, help="cap on the movers' grid (0 = fill the GPU)")
@@ -669,8 +829,13 @@ def main():
     ap.add_argument("--requests", type=int, default=0, help="override the request count")
     ap.add_argument("--fixed-tokens", type=int, default=0, help="give every request this many tokens")
     ap.add_argument("--low-latency", action="store_true", help="batched resume with KVR_LOW_LATENCY")
+    ap.add_argument("--no-share", action="store_true", help="paper_shape: every request owns its whole context")
     ap.add_argument("--no-extras", action="store_true", help="skip kernels-alone, lone-request and CPU legs")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="launcher and bookkeeping check without a GPU: metadata-only pools, gloo ranks; moves nothing")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(relaunch_under_torchrun(args))
     if args.impl == "reference":
         run_reference(args)
     elif args.workload == "longctx":

@@ -43,8 +43,17 @@
  *     blocks or host bytes are ordered after the move on the device, so the
  *     caller never has to wait for correctness of the library's own moves;
  *   - calls on one pool may come from any thread: they are serialised by a lock inside the pool and make the
- *     pool's device current for their duration (kvr_wait only takes the lock to look, not while it sleeps).
- *     kvr_pool_destroy must not race with other calls.  A kvr_controller is single-threaded.
+ *     pool's device current for their duration.  Whenever a call has to wait on the host for GPU work (kvr_wait,
+ *     KVR_SYNC, an expire / release / admit that meets a move in flight, a move call that finds every descriptor
+ *     buffer taken) it gives the lock up while it sleeps, so other threads keep working on the pool.
+ *     kvr_pool_destroy must not race with other calls.  A kvr_controller is single-threaded;
+ *   - a move call that fails while enqueueing (a CUDA error, out of host memory) leaves every request of the batch
+ *     exactly as it was: states, block tables, free-queue order, arena ranges and counters are restored, GPU work
+ *     already queued for it is waited for, and each affected per_req entry carries the error;
+ *   - nothing is allocated on the move path: streams, events of the staging ring, staging memory and the
+ *     descriptor buffers (max_moves_in_flight of them, each large enough for the block tables of the whole pool)
+ *     exist from kvr_pool_create on.  The one exception is a move whose descriptors exceed such a buffer (tens of
+ *     thousands of chunk pieces): it takes a one-off buffer that is freed when the move retires.
  */
 #ifndef KVR_H
 #define KVR_H
@@ -85,6 +94,8 @@ enum {
 #define KVR_METADATA_ONLY 1u         /* bookkeeping only: no buffers, no CUDA calls, nothing moves */
 #define KVR_PROFILE 2u               /* bracket every mover launch with timing events (gather_ms, scatter_ms) */
 
+#define KVR_ROUTE_AUTO 0             /* staged (the measured winner on B200); mapped when no staging memory can be had
+                                        (neither the caller's nor an allocation) and the arena is mapped host memory */
 #define KVR_ROUTE_STAGED 1           /* kernel <-> HBM staging ring <-> chunked cudaMemcpyAsync */
 #define KVR_ROUTE_MAPPED 2           /* kernel reads / writes the pinned arena directly over the host link */
 #define KVR_ROUTE_DMA2D 3            /* no kernel: one strided cudaMemcpy2DAsync per block, pool <-> arena */
@@ -105,9 +116,13 @@ typedef struct {
   int32_t num_blocks;
   int32_t device;                    /* CUDA device ordinal */
   uint64_t host_capacity_bytes;      /* host tier budget */
-  uint64_t chunk_bytes;              /* staging slot size = largest chunk, multiple of 4096; 0 = 512 MiB */
-  int32_t staging_slots;             /* slots per direction, >= 2; 0 = 2 */
-  int32_t route;                     /* KVR_ROUTE_*; 0 = KVR_ROUTE_STAGED */
+  uint64_t chunk_bytes;              /* staging slot size: the granule in which staging memory is reused and the
+                                        largest single copy over the link; multiple of 4096, at least one tile;
+                                        0 = 64 MiB */
+  int32_t staging_slots;             /* slots per direction, in [2, 64]; 0 = 16.  Staging memory is one ring of
+                                        staging_slots x chunk_bytes per direction (default 2 x 1 GiB); one mover
+                                        launch covers up to staging_slots - 1 consecutive slots of its ring */
+  int32_t route;                     /* KVR_ROUTE_* */
   int32_t kernel;                    /* KVR_KERNEL_*; 0 = KVR_KERNEL_BULK */
   int32_t max_ctas;                  /* cap on the movers' grid (0 = fill the GPU) */
   uint32_t flags;                    /* KVR_METADATA_ONLY | KVR_PROFILE */
@@ -120,10 +135,32 @@ typedef struct {
                                         access enabled): the tier then lives in HBM and images are device
                                         memory; with KVR_ROUTE_MAPPED the movers write it directly */
   const int32_t *initial_free_order; /* permutation of [0, num_blocks) or NULL = 0, 1, 2, ... */
+  /* Everything below may be left zero. */
+  void *device_staging;              /* DEVICE pointer to 2 x staging_slots x chunk_bytes bytes, 256-byte aligned
+                                        (an engine that owns all of HBM carves it out of its own memory), or NULL:
+                                        the library allocates it at pool creation */
+  void *streams[4];                  /* cudaStream_t for the gather kernel, the device-to-host copies, the
+                                        host-to-device copies and the scatter kernel, in that order; four distinct
+                                        streams of cfg->device, or NULL each: the library creates high-priority
+                                        non-blocking streams.  Caller-owned streams must not be used for anything
+                                        that waits on this pool's moves from inside the same stream */
+  uint64_t ramp_start_bytes;         /* a move of up to this many bytes is one mover launch; a larger one keeps the
+                                        first launch of a suspend and the last launch of a resume down to one slot
+                                        (so the link starts at once and little scattering remains after the last
+                                        byte) and makes every other launch as large as the ring allows.
+                                        0 = 256 MiB: 85 us of mover time */
+  uint64_t copy_piece_bytes;         /* link copies are issued in pieces of at most this size (and never across a
+                                        staging slot unless it is larger than a slot); 0 = 64 MiB */
+  int32_t max_moves_in_flight;       /* descriptor buffers created with the pool, one per move in flight, in
+                                        [1, 256]; 0 = 16.  A move call waits (bounded) while all are taken */
+  int32_t bulk_warps, bulk_stages, bulk_piece_bytes;   /* shape of the bulk mover: pipelines per CTA (1..8),
+                                        shared-memory stages per pipeline (2, 3, 4, 6 or 8), bytes per bulk copy
+                                        (multiple of 16); all three 0 = chosen from the tile size */
 } kvr_config;
 
 typedef struct {
-  int64_t blocks_total, blocks_free, blocks_active, blocks_pinned;
+  int64_t blocks_total, blocks_free, blocks_active, blocks_pinned;   /* distinct blocks: pinned = named by a RETAINED
+                                                     request or by the kept prefix of a HOST request; active = held otherwise */
   uint64_t host_capacity, host_used, host_largest_hole;
   int64_t n_active, n_retained, n_host, n_expired;
   int64_t suspends, resumes, resident_resumes, expires, recompute_marked;
@@ -174,8 +211,31 @@ kvr_status kvr_request_admit(kvr_pool *pool, uint64_t req_id, int64_t n_tokens, 
 /* Same, into blocks the caller names (an engine with its own allocator mirrors its choice): nb =
  * ceil(n_tokens/block_size) ids, each currently free, no repeats; the other free ids keep their order. */
 kvr_status kvr_request_admit_into(kvr_pool *pool, uint64_t req_id, int64_t n_tokens, const int32_t *blocks, int32_t nb);
-/* Forget a request in any state; its blocks go to the free tail, its host range is freed. */
+/* Forget a request in any state; its references to blocks are dropped (a block whose last reference goes joins the
+ * free tail), its host range is freed. */
 kvr_status kvr_request_release(kvr_pool *pool, uint64_t req_id);
+
+/*
+ * Shared prefix (Section 2, approval-gated workload: a system prefix shared through prefix caching, so that only
+ * the private suffix is per-request suspended state; Appendix B prices that suffix).  The new request's first
+ * n_shared_blocks logical blocks ARE the donor's first n_shared_blocks blocks, one more reference each; the rest
+ * come from the head of the free queue.  Blocks are reference counted: a block rejoins the free queue only when
+ * the last request naming it lets go, so a prefix lives exactly as long as somebody refers to it.  A request keeps
+ * referring to its shared prefix while it is RETAINED or on the HOST (the prefix stays resident and is counted in
+ * blocks_pinned); kvr_suspend_to_host moves only the private suffix -- tokens [n_shared_blocks * block_size,
+ * n_tokens), an image of (n_tokens - n_shared_blocks * block_size) * bytes_per_token bytes -- and a resume gives
+ * the request its old prefix followed by fresh blocks.
+ * Sharing is by whole blocks: n_shared_blocks * block_size tokens must lie inside the new request and inside the
+ * donor.  The donor may be ACTIVE or RETAINED (any of its full blocks) or on the HOST (its own shared prefix);
+ * with n_shared_blocks = 0 the donor is ignored and the call equals kvr_request_admit.
+ * KVR_HBM_FULL, KVR_ERR_BAD_STATE (id exists, donor EXPIRED), KVR_ERR_UNKNOWN_REQUEST (donor), KVR_ERR_INVALID_ARG.
+ */
+kvr_status kvr_request_admit_sharing(kvr_pool *pool, uint64_t req_id, int64_t n_tokens, uint64_t donor_id,
+                                     int32_t n_shared_blocks, int32_t *out_blocks, int32_t cap);
+/* The shared prefix a request refers to: its length in blocks and (cap entries, may be NULL) the ids. */
+kvr_status kvr_request_sharing(kvr_pool *pool, uint64_t req_id, int32_t *n_shared_blocks, int32_t *blocks, int32_t cap);
+/* Number of references to one block (0 = free); -1 for an id out of range. */
+int32_t kvr_block_refcount(kvr_pool *pool, int32_t block);
 
 /*
  * State 1 of Eq. 1 (Section 3.1): keep the KV in HBM.  ACTIVE -> RETAINED; the
@@ -215,8 +275,9 @@ kvr_status kvr_expire(kvr_pool *pool, const uint64_t *req, int32_t n, kvr_status
 kvr_status kvr_resume_from_host(kvr_pool *pool, const uint64_t *req, int32_t n, uint32_t flags, kvr_status *per_req);
 /*
  * Same move for one HOST request into blocks the caller names (each currently
- * free, no repeats, nb = its block count); the other free ids keep their
- * order.  This is how "any block relabelling" is exercised.
+ * free, no repeats, nb = its private block count: all of its blocks unless it
+ * shares a prefix); the other free ids keep their order.  This is how "any
+ * block relabelling" is exercised.
  */
 kvr_status kvr_resume_from_host_into(kvr_pool *pool, uint64_t req, const int32_t *blocks, int32_t nb, uint32_t flags);
 
@@ -297,7 +358,8 @@ kvr_status kvr_read_load(const void *device_buf, uint64_t bytes, int32_t launche
 /*
  * The copy benchmark behind the host-resume price beta_2 (Appendix B: one contiguous payload between page-locked
  * host memory and the device, synchronised before and after, repeated): copies `bytes` (clipped to the arena)
- * between the pool's own arena and a temporary device buffer, reps times each way after two warm-ups, and reports
+ * between the pool's own arena and the pool's staging memory (a temporary device buffer only when `bytes` exceeds
+ * it or the pool has none), reps times each way after two warm-ups, and reports
  * the best rate per direction in GB/s (1e9).  This is the link roofline the moves are judged against, measured
  * on the very memory they use.  The arena must hold no image (KVR_ERR_BAD_STATE otherwise): it is overwritten.
  */
@@ -311,6 +373,15 @@ kvr_status kvr_probe_link(kvr_pool *pool, uint64_t bytes, int32_t reps, double *
  * stays set so that the reporting through kvr_wait() can be observed; kvr_clear_device_error() resets it.
  */
 kvr_status kvr_selftest_bounded_wait(kvr_pool *pool, int32_t leave_error_set);
+/*
+ * Self-test of the movers' table check (no counterpart in the paper).  Every block table is validated on the host
+ * before it is uploaded; the kernels check each entry once more against the pool's block count, skip a tile whose
+ * entry is out of range and write 3 to the device-error word, so the pool is never addressed outside its extent.
+ * This call makes the check fire safely: it launches the gather over one tile whose entry names the pool's last
+ * block while telling the kernel that the pool is one block shorter (the entry is out of range for the kernel, yet
+ * inside the real allocation).  KVR_OK means the tile was skipped and the word was written.
+ */
+kvr_status kvr_selftest_block_check(kvr_pool *pool, int32_t leave_error_set);
 kvr_status kvr_clear_device_error(kvr_pool *pool);
 
 kvr_status kvr_pool_stats(kvr_pool *pool, kvr_stats *out);
@@ -380,6 +451,29 @@ kvr_status kvr_controller_advance(kvr_controller *c, double now, int32_t *n_offl
  * prefills), KVR_HBM_FULL (nothing changed; free blocks and call again) */
 kvr_status kvr_controller_resume(kvr_controller *c, uint64_t req, double now);
 kvr_status kvr_controller_get_stats(kvr_controller *c, kvr_controller_stats *out);
+
+/*
+ * Host-made failures for tests (no counterpart in the paper; nothing here touches the GPU).  kind 0: the n-th CUDA
+ * runtime call a move makes from now on (event record, stream wait, copy, kernel launch, ...) reports failure
+ * WITHOUT being issued; kind 1: the n-th host allocation point of the move path throws as if memory had run out.
+ * n = 0 disarms.  kvr_test_points() returns how many such points were passed since the last arming, so a test can
+ * walk n over a whole move.
+ */
+#define KVR_FAIL_CUDA 0
+#define KVR_FAIL_ALLOC 1
+kvr_status kvr_test_fail_nth(kvr_pool *pool, int32_t kind, int64_t n);
+int64_t kvr_test_points(kvr_pool *pool, int32_t kind);
+
+/*
+ * Placement of the library's own arena (no counterpart in the paper).  Host DRAM is shared between the GPUs of a
+ * node; each pool's arena is faulted in by threads bound to the CPUs of the NUMA node its GPU hangs off, so the
+ * pages land next to that GPU's link.  kvr_pool_numa_node: the node used (-1: unknown, single-node host, caller's
+ * arena).  kvr_numa_lookup: the parsing on its own -- node of the PCI device `pci_bus_id` ("0000:1b:00.0") and the
+ * CPUs of that node under `sysfs_root` (NULL = "/sys"); returns the CPU count (cpus: cap entries, may be NULL),
+ * *node = -1 and 0 when the tree does not say.
+ */
+int32_t kvr_pool_numa_node(kvr_pool *pool);
+int32_t kvr_numa_lookup(const char *sysfs_root, const char *pci_bus_id, int32_t *node, int32_t *cpus, int32_t cap);
 
 /* copies the free queue, head first, into out (cap entries, may be NULL); returns its length */
 int64_t kvr_free_queue(kvr_pool *pool, int32_t *out, int64_t cap);

@@ -46,6 +46,11 @@ CONFIGS = {
     "paper_70b_tp4": Workload("paper_70b_tp4", 80, 2, 128, 2, 16, 32768, 32,
                               ("lognormal", 8192, 0.6, 1024, 32768), occupancy=0.70,
                               notes="per-GPU KV shard of the paper's serving setup; small tiles"),
+    # not one of the five either: the paper's workload shape on that rank -- a median gate context of 8.4K tokens of
+    # which a 5.4K-token system prefix is shared by every request and ~3.0K tokens are private (Section 2)
+    "paper_shape": Workload("paper_shape", 80, 2, 128, 2, 16, 32768, 32, ("fixed", 8400), occupancy=0.50,
+                            notes="32 gate contexts of 8,400 tokens sharing one 5,400-token prefix",
+                            extra={"shared_tokens": 5400}),
 }
 
 

@@ -6,7 +6,8 @@ The rules, in the paper's words restated (Section 3.4; Appendix D, live-controll
   * under the cpu_ttl(lambda) branch it then carries a one-shot timer t_2(lambda); when it fires before the
     resume, the host copy is discarded and the context is never re-scored;
   * a full host tier rejects the newcomer (replay rule: residents are never displaced) or, under the live rule,
-    first discards the copy that has been suspended longest;
+    makes room by priority: first a copy whose timer has already run out, then the copy that has been suspended
+    longest (the class in between, transient blocks of active requests, cannot occur in a tier of suspended contexts);
   * a resume costs 0 from HBM plus alpha_1 per second it was pinned there, beta_2 from the host copy, beta_3
     otherwise (Eq. 1).
 Everything is linear scans over a dictionary: no heaps, no sets, no shared code with the library.
@@ -48,6 +49,17 @@ class OrcController:
             if st == orc.OK:
                 break
             assert st == orc.HOST_FULL, st
+            # live rule (Appendix D): evict by priority.  First, copies whose timer has already run out at this
+            # instant (due at the same time as this offload, not fired yet); the paper's second class -- transient
+            # blocks of active requests -- does not exist in a host tier that holds suspended contexts only; then
+            # the copy that has been suspended longest.
+            expired = [(v[2], k) for k, v in self.ctx.items() if v[0] == ON_HOST and v[2] <= self.now]
+            if self.admission == LIVE and expired:
+                _, victim = min(expired)
+                assert self.pool.expire([victim])[0] == orc.OK
+                self.ctx[victim][0], self.ctx[victim][2] = GONE, math.inf
+                self.st["ttl_expired"] += 1
+                continue
             on_host = [(v[1], k) for k, v in self.ctx.items() if v[0] == ON_HOST]
             if self.admission == LIVE and on_host:
                 _, victim = min(on_host)                      # suspended longest

@@ -49,7 +49,26 @@ struct kvr_controller {
       kvr_status s = kvr_suspend_to_host(pool, &id, 1, 0, nullptr);
       if (s == KVR_OK) break;
       if (s != KVR_HOST_FULL) return s;
-      // live rule: make room by discarding the least recently suspended host copy; replay rule: never displace
+      // live rule, first class (Appendix D: "blocks whose timer has expired" go first): a host copy whose one-shot
+      // timer has run out by this instant but has not been fired yet (it is due at the very same time as this
+      // offload) is discarded before any copy that is still within its timer
+      if (cfg.admission == KVR_ADMIT_LIVE) {
+        uint64_t due = 0;
+        bool found = false;
+        for (auto it = timers.begin(); it != timers.end() && it->first <= now; ++it)
+          if (ctx[it->second].where == ON_HOST) { due = it->second; found = true; break; }
+        if (found) {
+          Ctx &v = ctx[due];
+          kvr_status e = kvr_expire(pool, &due, 1, nullptr);
+          if (e != KVR_OK) return e;
+          to_gone(due, v);
+          st.ttl_expired++;
+          continue;
+        }
+      }
+      // the paper's second class, transient blocks of active requests, has no counterpart here: the host tier holds
+      // images of suspended contexts only.  Third class: the least recently suspended host copy.
+      // Replay rule: never displace.
       if (cfg.admission == KVR_ADMIT_LIVE && !lru.empty()) {
         const uint64_t victim = lru.begin()->second;
         Ctx &v = ctx[victim];

@@ -74,6 +74,13 @@ __device__ __forceinline__ Tile locate(const MoveArgs &a, const long long *cum, 
   long long valid = sg.n_tokens - first_tok;
   if (valid > a.block_size) valid = a.block_size;
   Tile t;
+  // The host validates every table before it is uploaded; should an entry still arrive out of range, the tile is
+  // skipped and the error word says so -- the pool is never addressed outside its extent.
+  if (a.num_blocks > 0 && (unsigned)blk >= (unsigned)a.num_blocks) {
+    if (a.status) { *reinterpret_cast<volatile int *>(a.status) = kStatusBadBlock; __threadfence_system(); }
+    t.pool_ptr = a.pool; t.lin_ptr = sg.img; t.bytes = 0;
+    return t;
+  }
   t.pool_ptr = a.pool + plane * a.plane_stride + (long long)blk * a.block_stride;
   t.lin_ptr = sg.img + (plane * sg.n_tokens + first_tok) * a.row_bytes;
   t.bytes = (int)valid * a.row_bytes;

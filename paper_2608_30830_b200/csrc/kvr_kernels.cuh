@@ -32,7 +32,8 @@ struct MoveArgs {
   int tile_bytes;        // block_size * row_bytes
   int row_bytes;         // kv_heads * head_dim * dtype_bytes (multiple of 16)
   int block_size;
-  int *status;           // DEVICE: error word (0 = fine), written only when a bounded wait runs out
+  int num_blocks;        // blocks in the pool: a table entry outside [0, num_blocks) is never dereferenced (0 = unchecked)
+  int *status;           // DEVICE or NULL: error word (0 = fine); 1 = a bounded wait ran out, 3 = a table entry out of range
   unsigned long long *stamp;  // DEVICE or NULL: stamp[0] = earliest start, stamp[1] = latest end of any CTA, in
                               // %globaltimer nanoseconds (the host initialises them to ~0 and 0)
 };
@@ -54,5 +55,7 @@ cudaError_t launch_read_load(const void *buf, unsigned long long bytes, int laun
 
 // one thread waits `limit` polls on an mbarrier nobody completes, then writes 2 to *status (pinned host word)
 cudaError_t launch_wait_limit_probe(int *status, unsigned limit, cudaStream_t s);
+
+constexpr int kStatusWaitRanOut = 1, kStatusProbe = 2, kStatusBadBlock = 3;
 
 }  // namespace kvr

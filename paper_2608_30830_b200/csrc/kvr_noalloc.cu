@@ -126,6 +126,7 @@ extern "C" kvr_status kvr_gather_noalloc(const void *device_pool, const kvr_geom
   a.block_stride = (long long)tile;
   a.row_bytes = (int)row;
   a.block_size = g->block_size;
+  a.num_blocks = num_blocks;
   a.status = nullptr;               // the warp mover has no bounded waits and never writes it
   cudaError_t e = kvr::launch_move_warp(true, a, 0, g_sm_count[dev], st);
   if (e != cudaSuccess) return fail_na(KVR_ERR_CUDA, cudaGetErrorString(e));

@@ -13,7 +13,8 @@ ACTIVE, RETAINED, SUSPENDING, HOST, RESUMING, EXPIRED = 0, 1, 2, 3, 4, 5
 SYNC = 1
 LOW_LATENCY = 2
 METADATA_ONLY, PROFILE = 1, 2
-ROUTE_STAGED, ROUTE_MAPPED, ROUTE_DMA2D = 1, 2, 3
+ROUTE_AUTO, ROUTE_STAGED, ROUTE_MAPPED, ROUTE_DMA2D = 0, 1, 2, 3
+FAIL_CUDA, FAIL_ALLOC = 0, 1
 LAYER_MAJOR, BLOCK_MAJOR = 0, 1
 KERNEL_WARP, KERNEL_BULK = 1, 2
 ALL = 2**64 - 1
@@ -35,7 +36,11 @@ class Config(C.Structure):
                 ("staging_slots", C.c_int32), ("route", C.c_int32), ("kernel", C.c_int32),
                 ("max_ctas", C.c_int32), ("flags", C.c_uint32), ("layout", C.c_int32),
                 ("device_pool", C.c_void_p), ("host_arena", C.c_void_p),
-                ("initial_free_order", C.POINTER(C.c_int32))]
+                ("initial_free_order", C.POINTER(C.c_int32)),
+                ("device_staging", C.c_void_p), ("streams", C.c_void_p * 4),
+                ("ramp_start_bytes", C.c_uint64), ("copy_piece_bytes", C.c_uint64),
+                ("max_moves_in_flight", C.c_int32), ("bulk_warps", C.c_int32), ("bulk_stages", C.c_int32),
+                ("bulk_piece_bytes", C.c_int32)]
 
 
 class Prices(C.Structure):
@@ -71,10 +76,12 @@ class Stats(C.Structure):
 
 EXPORTS = [
     "kvr_bytes_per_token", "kvr_pool_create", "kvr_pool_destroy", "kvr_request_admit", "kvr_request_admit_into", "kvr_request_release",
+    "kvr_request_admit_sharing", "kvr_request_sharing", "kvr_block_refcount", "kvr_test_fail_nth", "kvr_test_points",
+    "kvr_pool_numa_node", "kvr_numa_lookup",
     "kvr_retain_in_hbm", "kvr_suspend_to_host", "kvr_expire", "kvr_resume_from_host",
     "kvr_resume_from_host_into", "kvr_export_to_device", "kvr_import_from_device", "kvr_request_info",
     "kvr_request_latency", "kvr_wait", "kvr_pool_stats", "kvr_free_queue", "kvr_pool_device_ptr",
-    "kvr_pool_host_arena", "kvr_last_error", "kvr_gather_noalloc", "kvr_read_load", "kvr_probe_link", "kvr_selftest_bounded_wait", "kvr_clear_device_error",
+    "kvr_pool_host_arena", "kvr_last_error", "kvr_gather_noalloc", "kvr_read_load", "kvr_probe_link", "kvr_selftest_bounded_wait", "kvr_selftest_block_check", "kvr_clear_device_error",
     "kvr_policy_break_evens", "kvr_policy_host_ttl", "kvr_policy_replay", "kvr_policy_select",
     "kvr_controller_create", "kvr_controller_destroy", "kvr_controller_calibrate", "kvr_controller_suspend",
     "kvr_controller_advance", "kvr_controller_resume", "kvr_controller_get_stats",
@@ -109,6 +116,20 @@ def lib():
     L.kvr_request_admit_into.argtypes = [vp, u64, i64, pi32, i32]
     L.kvr_request_release.restype = i32
     L.kvr_request_release.argtypes = [vp, u64]
+    L.kvr_request_admit_sharing.restype = i32
+    L.kvr_request_admit_sharing.argtypes = [vp, u64, i64, u64, i32, pi32, i32]
+    L.kvr_request_sharing.restype = i32
+    L.kvr_request_sharing.argtypes = [vp, u64, pi32, pi32, i32]
+    L.kvr_block_refcount.restype = i32
+    L.kvr_block_refcount.argtypes = [vp, i32]
+    L.kvr_test_fail_nth.restype = i32
+    L.kvr_test_fail_nth.argtypes = [vp, i32, i64]
+    L.kvr_test_points.restype = i64
+    L.kvr_test_points.argtypes = [vp, i32]
+    L.kvr_pool_numa_node.restype = i32
+    L.kvr_pool_numa_node.argtypes = [vp]
+    L.kvr_numa_lookup.restype = i32
+    L.kvr_numa_lookup.argtypes = [C.c_char_p, C.c_char_p, pi32, pi32, i32]
     for name in ("kvr_retain_in_hbm", "kvr_expire"):
         f = getattr(L, name)
         f.restype = i32
@@ -164,6 +185,8 @@ def lib():
     L.kvr_controller_get_stats.argtypes = [vp, C.POINTER(ControllerStats)]
     L.kvr_selftest_bounded_wait.restype = i32
     L.kvr_selftest_bounded_wait.argtypes = [vp, i32]
+    L.kvr_selftest_block_check.restype = i32
+    L.kvr_selftest_block_check.argtypes = [vp, i32]
     L.kvr_clear_device_error.restype = i32
     L.kvr_clear_device_error.argtypes = [vp]
     L.kvr_probe_link.restype = i32
@@ -272,6 +295,15 @@ def read_load(device_buf, nbytes, launches, device_sink, stream=None):
     return lib().kvr_read_load(device_buf, nbytes, launches, device_sink, stream)
 
 
+def numa_lookup(sysfs_root, pci_bus_id, cap=4096):
+    """kvr_numa_lookup: (node, [cpus]) of a PCI device under a sysfs tree (None = the machine's /sys)."""
+    node = C.c_int32()
+    cpus = np.zeros(cap, dtype=np.int32)
+    n = lib().kvr_numa_lookup(None if sysfs_root is None else str(sysfs_root).encode(), pci_bus_id.encode(),
+                              C.byref(node), cpus.ctypes.data_as(C.POINTER(C.c_int32)), cap)
+    return node.value, cpus[:min(n, cap)].tolist()
+
+
 NOALLOC_MAX_BLOCKS = 65536
 
 
@@ -298,7 +330,8 @@ class Pool:
 
     def __init__(self, layers, kv_heads, head_dim, dtype_bytes, block_size, num_blocks, host_capacity_bytes,
                  initial_free_order=None, device=0, chunk_bytes=0, staging_slots=0, route=0, kernel=0,
-                 max_ctas=0, flags=0, device_pool=None, host_arena=None, layout=0):
+                 max_ctas=0, flags=0, device_pool=None, host_arena=None, layout=0, device_staging=None, streams=None,
+                 ramp_start_bytes=0, copy_piece_bytes=0, max_moves_in_flight=0, bulk_shape=None):
         self.geom = (layers, kv_heads, head_dim, dtype_bytes, block_size)
         self.NB = num_blocks
         cfg = Config()
@@ -309,6 +342,15 @@ class Pool:
         self.layout = layout
         cfg.device_pool = device_pool
         cfg.host_arena = host_arena
+        cfg.device_staging = device_staging
+        if streams is not None:
+            if len(streams) != 4:
+                raise ValueError("streams: gather, d2h, h2d, scatter")
+            for i, st in enumerate(streams):
+                cfg.streams[i] = st
+        cfg.ramp_start_bytes, cfg.copy_piece_bytes, cfg.max_moves_in_flight = ramp_start_bytes, copy_piece_bytes, max_moves_in_flight
+        if bulk_shape is not None:
+            cfg.bulk_warps, cfg.bulk_stages, cfg.bulk_piece_bytes = bulk_shape
         order = None
         if initial_free_order is not None:
             order = np.ascontiguousarray(initial_free_order, dtype=np.int32)
@@ -353,6 +395,35 @@ class Pool:
 
     def release(self, rid):
         return lib().kvr_request_release(self._h, rid)
+
+    def admit_sharing(self, rid, n_tokens, donor, n_shared):
+        nb = max(0, -(-n_tokens // self.geom[4]))
+        out = np.zeros(max(nb, 1), dtype=np.int32)
+        st = lib().kvr_request_admit_sharing(self._h, rid, n_tokens, donor, n_shared, _i32p(out), nb)
+        return st, (out[:nb].copy() if st == OK else None)
+
+    def sharing(self, rid):
+        """(status, shared-prefix block ids the request refers to)."""
+        ns = C.c_int32()
+        st = lib().kvr_request_sharing(self._h, rid, C.byref(ns), None, 0)
+        if st != OK:
+            return st, None
+        out = np.zeros(max(ns.value, 1), dtype=np.int32)
+        lib().kvr_request_sharing(self._h, rid, None, _i32p(out), ns.value)
+        return st, out[:ns.value].copy()
+
+    def refcount(self, blk):
+        return int(lib().kvr_block_refcount(self._h, blk))
+
+    def test_fail_nth(self, kind, n):
+        return lib().kvr_test_fail_nth(self._h, kind, n)
+
+    def test_points(self, kind):
+        return int(lib().kvr_test_points(self._h, kind))
+
+    @property
+    def numa_node(self):
+        return int(lib().kvr_pool_numa_node(self._h))
 
     # -- the named calls
     def _batch(self, fn, ids, *flags):
@@ -433,6 +504,9 @@ class Pool:
 
     def selftest_bounded_wait(self, leave_error_set=False):
         return lib().kvr_selftest_bounded_wait(self._h, int(leave_error_set))
+
+    def selftest_block_check(self, leave_error_set=False):
+        return lib().kvr_selftest_block_check(self._h, int(leave_error_set))
 
     def clear_device_error(self):
         return lib().kvr_clear_device_error(self._h)

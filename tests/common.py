@@ -10,14 +10,21 @@ COMMON_STATS = ["blocks_total", "blocks_free", "blocks_active", "blocks_pinned",
                 "bytes_suspended", "bytes_resumed", "bytes_expired_from_host"]
 
 
-def random_script(seed, n_ops, max_tokens, n_ids=12, batch=4):
-    """A seeded list of calls over a small id space; illegal calls are included on purpose."""
+def random_script(seed, n_ops, max_tokens, n_ids=12, batch=4, sharing=False):
+    """A seeded list of calls over a small id space; illegal calls are included on purpose.  With sharing=True
+    some admissions name a donor and a number of shared prefix blocks (often illegal ones, on purpose)."""
     rng = np.random.default_rng(seed)
     ops = []
+    kinds = ["admit", "admit", "admit_into", "retain", "suspend", "suspend", "expire", "resume", "resume",
+             "resume_into", "release"]
+    if sharing:
+        kinds += ["admit_sharing", "admit_sharing", "admit_sharing"]
     for _ in range(n_ops):
-        kind = rng.choice(["admit", "admit", "admit_into", "retain", "suspend", "suspend", "expire", "resume", "resume",
-                           "resume_into", "release"])
-        if kind == "admit":
+        kind = rng.choice(kinds)
+        if kind == "admit_sharing":
+            ops.append(("admit_sharing", int(rng.integers(n_ids)), int(rng.integers(0, max_tokens + 1)),
+                        int(rng.integers(n_ids)), int(rng.integers(0, 5))))
+        elif kind == "admit":
             ops.append(("admit", int(rng.integers(n_ids)), int(rng.integers(0, max_tokens + 1))))
         elif kind == "admit_into":
             ops.append(("admit_into", int(rng.integers(n_ids)), int(rng.integers(0, max_tokens + 1)), int(rng.integers(2**31))))
@@ -41,9 +48,11 @@ def snapshot(pool, ids):
         # transient states settle to these
         state = {2: 3, 4: 0}.get(state, state)
         reqs[rid] = (state, d["n_tokens"], d["nb"], d["image_bytes"], d["arena_offset"],
-                     None if d["blocks"] is None else d["blocks"].tolist())
+                     None if d["blocks"] is None else d["blocks"].tolist(), pool.sharing(rid)[1].tolist())
     s = pool.stats()
-    return reqs, pool.free_queue().tolist(), {k: int(s[k]) for k in COMMON_STATS}
+    fq = pool.free_queue().tolist()
+    counts = [pool.refcount(b) for b in range(s["blocks_total"])] if s["blocks_total"] <= 4096 else None
+    return reqs, fq, {k: int(s[k]) for k in COMMON_STATS}, counts
 
 
 def run_script(pool, ops, n_ids=12, after_each=None):
@@ -54,6 +63,9 @@ def run_script(pool, ops, n_ids=12, after_each=None):
         per = None
         if kind == "admit":
             st, blocks = pool.admit(op[1], op[2])
+            per = None if blocks is None else blocks.tolist()
+        elif kind == "admit_sharing":
+            st, blocks = pool.admit_sharing(op[1], op[2], op[3], op[4])
             per = None if blocks is None else blocks.tolist()
         elif kind == "admit_into":
             bs = pool.geom[4]
@@ -68,7 +80,7 @@ def run_script(pool, ops, n_ids=12, after_each=None):
         elif kind == "resume_into":
             s0, d = pool.info(op[1])
             fq = pool.free_queue()
-            nb = d["nb"] if s0 == orc.OK else 1
+            nb = d["nb"] - len(pool.sharing(op[1])[1]) if s0 == orc.OK else 1     # the private part is what moves
             pick = np.random.default_rng(op[2]).permutation(fq)[:nb]
             if len(pick) < nb:                       # not enough free blocks: name an invalid list
                 pick = np.concatenate([pick, np.zeros(nb - len(pick), dtype=np.int32) - 1])
@@ -84,22 +96,26 @@ def run_script(pool, ops, n_ids=12, after_each=None):
 
 
 def check_invariants(pool, ids):
-    """Pool conservation, disjointness and host accounting (properties, valid for either implementation)."""
+    """Pool conservation, reference counts and host accounting (properties, valid for either implementation)."""
     s = pool.stats()
-    seen = list(pool.free_queue())
-    held = host = 0
+    fq = list(pool.free_queue())
+    refs = np.zeros(s["blocks_total"], dtype=np.int64)
+    host = 0
     for rid in ids:
         st, d = pool.info(rid)
         if st != orc.OK:
             continue
         state = {2: 3, 4: 0}.get(d["state"], d["state"])
         if state in (orc.ACTIVE, orc.RETAINED):
-            seen += list(d["blocks"])
-            held += d["nb"]
+            np.add.at(refs, d["blocks"], 1)
         if state == orc.HOST:
+            np.add.at(refs, pool.sharing(rid)[1], 1)                # the prefix a request on the host still refers to
             host += -(-d["image_bytes"] // 4096) * 4096
-    assert s["blocks_free"] + held == s["blocks_total"]
+    held = int((refs > 0).sum())
+    assert s["blocks_free"] + held == s["blocks_total"]             # free + distinct held = NB
     assert s["blocks_active"] + s["blocks_pinned"] == held
-    assert sorted(seen) == list(range(s["blocks_total"]))
+    assert sorted(fq) == np.flatnonzero(refs == 0).tolist()
+    if s["blocks_total"] <= 4096:
+        assert [pool.refcount(b) for b in range(s["blocks_total"])] == refs.tolist()
     assert s["host_used"] == host <= s["host_capacity"]
     assert s["bytes_suspended"] - s["bytes_resumed"] - s["bytes_expired_from_host"] >= 0

@@ -28,3 +28,18 @@ def test_other_ranks_of_the_reference_arm_stay_silent():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
                           "--warmup", "1"], capture_output=True, text=True, timeout=120, env=env)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_plain_launch_with_gpus_2_starts_two_ranks_and_prints_one_line():
+    """`python bench.py --gpus 2` with no launcher in the environment must start the ranks itself.  Checked without a
+    GPU through --dry-run: metadata-only pools, gloo ranks, the same barriers and reductions, one line from rank 0."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run", "--steps", "2",
+                          "--warmup", "1", "--workload", "paper_shape"], capture_output=True, text=True, timeout=600, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [x for x in out.stdout.splitlines() if x.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["dry_run"] is True and d["value"] is None and d["scaling"] == "weak"
+    # 32 contexts of 8,400 tokens sharing 337 whole blocks (5,392 tokens): 3,008 private tokens each, on both ranks
+    assert d["bookkeeping"]["bytes_suspended_per_step_all_ranks"] == 2 * 32 * 3008 * 80 * 2 * 128 * 2 * 2

@@ -73,6 +73,42 @@ def test_live_admission_evicts_the_longest_suspended_by_hand():
     assert s["evicted_lru"] == 1 and s["gpu_cost"] == pytest.approx(1.91 + 0.02 + 0.02)
 
 
+def test_live_admission_discards_an_expired_timer_before_any_lru_victim_by_hand():
+    """Appendix D, live rule: "blocks whose timer has expired" are evicted before least-recently-used suspended
+    blocks.  Worked by hand with exact numbers: prices (0.5, 1, 3), C2 = 3, W_ref = 96, lambda = 5/32 give
+    alpha_2 = 1/8 and t_2 = 16 s; grace 10 s.  X and W go to the host under host-retain (no timers); after the
+    branch is frozen to cpu_ttl, Y is offloaded at 24 (timer due at 40) and Z's offload falls due at 40 as well.
+    The tier is full at that instant: Y's timer has run out, so Y goes -- not X, which has been suspended longest."""
+    prices, c2, w_ref, lam = (0.5, 1.0, 3.0), 3, 96.0, 5.0 / 32.0
+    cal_arrive = [0, 1, 2, 30, 31, 32, 40, 41, 42]
+    cal_wait = [1000.0] * 3 + [1.0] * 6              # host-retain: 3 b2 + 6 b3 = 21; cpu_ttl: 3 b3 + 6 b2 = 15 -> cpu_ttl
+    po = orc.OrcPool(*GEOM, 64, 3 * 4096, with_data=False)
+    pg = kvr.Pool(*GEOM, 64, 3 * 4096, flags=kvr.METADATA_ONLY)
+    co = OrcController(po, prices, lam, w_ref, c2=c2, hbm_grace_s=10.0, branch=RETAIN, admission=LIVE)
+    cg = kvr.Controller(pg, prices, lam, w_ref, c2=c2, hbm_grace_s=10.0, branch=kvr.BRANCH_RETAIN, admission=kvr.ADMIT_LIVE)
+    X, W, Y, Z = 9, 7, 8, 1
+    for pool, ctl in ((po, co), (pg, cg)):
+        assert ctl.stats()["t2"] == 16.0
+        for rid in (X, W, Y, Z):
+            assert pool.admit(rid, 60)[0] == orc.OK
+        assert ctl.suspend(X, 0.0) == orc.RESIDENT and ctl.suspend(W, 1.0) == orc.RESIDENT
+        assert ctl.advance(12.0) == (orc.OK, 2, 0)                      # both on the host, no timers
+        assert ctl.calibrate(cal_arrive, cal_wait) == TTL
+        assert ctl.suspend(Y, 14.0) == orc.RESIDENT
+        assert ctl.advance(25.0) == (orc.OK, 1, 0)                      # Y on the host since 24, timer due at 40
+        assert ctl.suspend(Z, 30.0) == orc.RESIDENT                     # offload due at 40 too
+        st, n_off, n_exp = ctl.advance(41.0)
+        assert (st, n_off) == (orc.OK, 1)
+        states = {rid: pool.info(rid)[1]["state"] for rid in (X, W, Y, Z)}
+        assert states == {X: orc.HOST, W: orc.HOST, Y: orc.EXPIRED, Z: orc.HOST}
+        s = ctl.stats()
+        assert s["ttl_expired"] == 1 and s["evicted_lru"] == 0 and s["not_admitted"] == 0
+        assert ctl.resume(Y, 42.0) == orc.RECOMPUTE and ctl.resume(X, 43.0) == orc.OK
+        # HBM time: X 10 s, W 10 s, Y 10 s, Z 10 s at alpha_1 = 0.5; one recompute, one host resume
+        assert ctl.stats()["gpu_cost"] == pytest.approx(0.5 * 40 + 3.0 + 1.0)
+    assert snapshot(po, [X, W, Y, Z]) == snapshot(pg, [X, W, Y, Z])
+
+
 def test_grace_period_timer_and_hbm_cost_by_hand():
     pool = orc.OrcPool(*GEOM, 64, 8 * 4096, with_data=False)
     lam = 2 * 4 / 100.0                                             # c2 = 4, w_ref = 100 -> t2 = (1.91-0.02)/1.91*100

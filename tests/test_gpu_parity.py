@@ -559,7 +559,7 @@ def test_low_latency_resume_completes_requests_one_by_one():
     in order, the first long before the last, none later than under the default plan (where requests that share a
     chunk finish together)."""
     geom = (8, 8, 128, 2, 16)                      # 32 KiB per token
-    t = Twin(geom, 512, 256 << 20, seed=29, chunk_bytes=256 << 20)
+    t = Twin(geom, 512, 256 << 20, seed=29, chunk_bytes=256 << 20, staging_slots=2)
     ids = [0, 1, 2, 3]
     for rid in ids:
         assert t.both("admit", rid, 1500)[1][0] == kvr.OK        # 47 MiB each: all four fit one 256 MiB chunk

@@ -198,3 +198,133 @@ def test_a_plain_c_program_can_drive_the_library(tmp_path):
     out = subprocess.check_output([str(exe)], text=True).split()
     # free queue after the flow: 0 1 3 4 6 5 2 7 -> admit takes 0 1 3; five blocks stay free
     assert out == ["5", "1", "0", "1", "3", "1.136", "108.5", "1781.2", "64"]
+
+
+# ---- shared prefixes, reference counts ------------------------------------------------------
+
+@pytest.mark.parametrize("seed", range(8))
+def test_sharing_scripts_match_the_oracle(seed):
+    """Scripts whose admissions name donors and shared-prefix lengths (legal and illegal): statuses, tables, kept
+    prefixes, reference counts, arena offsets, free-queue order and counters equal the oracle's after every call."""
+    NB, cap = 32, 8 * 4096
+    a, b = pair(NB, cap, seed)
+    ops = random_script(500 + seed, 500, max_tokens=40, sharing=True)
+    la = run_script(a, ops)
+    lb = run_script(b, ops, after_each=lambda op, st: check_invariants(b, range(12)))
+    shared_admissions = 0
+    for (op, sa, pa, snap_a), (_, sb, pb, snap_b) in zip(la, lb):
+        assert (sa, pa) == (sb, pb), op
+        assert snap_a == snap_b, op
+        shared_admissions += op[0] == "admit_sharing" and sa == orc.OK and op[4] > 0
+    assert shared_admissions > 0
+
+
+def test_paper_context_split_in_the_library(golden):
+    """Section 2 / Appendix B: an 8,400-token context whose 5,400-token system prefix is shared moves 3,000 tokens =
+    983,040,000 bytes (0.98 GB), not 2.75 GB; the prefix stays resident while any referrer waits on the host."""
+    L, H, D, e = (int(x) for x in golden["bpt_factors"])
+    p = kvr.Pool(L, H, D, e, 8, 4096, 8 << 30, flags=kvr.METADATA_ONLY)
+    assert p.admit(0, 5400)[0] == kvr.OK
+    for rid in (1, 2, 3):
+        assert p.admit_sharing(rid, 8400, 0, 675)[0] == kvr.OK
+    assert p.release(0) == kvr.OK                                           # the prefix outlives the request that made it
+    assert p.suspend_to_host([1, 2, 3])[0] == kvr.OK
+    s = p.stats()
+    assert s["bytes_suspended"] == 3 * 983_040_000 and s["blocks_pinned"] == 675 and s["blocks_free"] == 4096 - 675
+    assert p.refcount(int(p.sharing(1)[1][0])) == 3
+    assert p.expire([1])[0] == kvr.OK and p.release(2) == kvr.OK
+    assert p.stats()["blocks_pinned"] == 675                                # request 3 still refers to it
+    assert p.resume_from_host([3])[0] == kvr.OK and p.info(3)[1]["nb"] == 1050
+    assert p.release(3) == kvr.OK and p.stats()["blocks_free"] == 4096      # freed with the last referrer
+
+
+# ---- a move that cannot be enqueued leaves everything unchanged (host-made failures) -----------
+
+def full_snapshot(p, ids):
+    from common import snapshot
+    return snapshot(p, ids)
+
+
+def test_injected_allocation_failures_leave_a_metadata_pool_unchanged():
+    NB, cap = 32, 8 * 4096
+    order = np.random.default_rng(3).permutation(NB).astype(np.int32)
+
+    def fresh():
+        o = orc.OrcPool(*GEOM, NB, cap, initial_free_order=order, with_data=False)
+        g = kvr.Pool(*GEOM, NB, cap, initial_free_order=order, flags=kvr.METADATA_ONLY)
+        for pool in (o, g):
+            assert pool.admit(1, 13)[0] == 0 and pool.admit_sharing(2, 17, 1, 2)[0] == 0 and pool.admit(3, 5)[0] == 0
+            assert pool.retain_in_hbm([3])[0] == 0
+        return o, g
+    for call in ("suspend", "resume", "resume_into"):
+        o, g = fresh()
+        if call != "suspend":
+            assert o.suspend_to_host([1, 2, 3])[0] == g.suspend_to_host([1, 2, 3])[0] == kvr.OK
+        pick = g.free_queue()[[5, 2, 9]].astype(np.int32)                    # request 2's private part: 3 blocks
+        do = {"suspend": lambda pool: pool.suspend_to_host([1, 9, 2, 3])[0],
+              "resume": lambda pool: pool.resume_from_host([2, 1, 9, 3])[0],
+              "resume_into": lambda pool: pool.resume_from_host_into(2, pick)}[call]
+        # how many allocation points does the call pass?  (armed far away, then read the counter)
+        probe = fresh()[1]
+        if call != "suspend":
+            probe.suspend_to_host([1, 2, 3])
+        assert probe.test_fail_nth(kvr.FAIL_ALLOC, 10**9) == kvr.OK
+        do(probe)
+        n_points = probe.test_points(kvr.FAIL_ALLOC)
+        assert n_points >= 2
+        for k in range(1, n_points + 1):
+            before = full_snapshot(g, range(12))
+            assert g.test_fail_nth(kvr.FAIL_ALLOC, k) == kvr.OK
+            st = do(g)
+            assert st == kvr.ERR_NOMEM, (call, k, st)
+            assert g.test_fail_nth(kvr.FAIL_ALLOC, 0) == kvr.OK
+            assert full_snapshot(g, range(12)) == before, (call, k)
+            check_invariants(g, range(12))
+        # disarmed, the same call goes through, and the pool keeps agreeing with the oracle afterwards
+        assert do(g) == do(o)
+        ops = random_script(77, 50, max_tokens=40, sharing=True)
+        for (op, sa, pa, snap_a), (_, sb, pb, snap_b) in zip(run_script(o, ops), run_script(g, ops)):
+            assert (sa, pa) == (sb, pb) and snap_a == snap_b, (call, op)
+
+
+# ---- free queue: named blocks leave in O(1) -------------------------------------------------------
+
+def test_named_admission_costs_microseconds_at_the_largest_pool():
+    """Appendix A: pinning removes blocks from the doubly linked free queue in O(1).  At the long-context
+    configuration's 147,456 blocks a named admission of 64 blocks must not scan the queue."""
+    import time
+    NB = 147456
+    p = kvr.Pool(32, 8, 128, 2, 8, NB, 0, flags=kvr.METADATA_ONLY)
+    rng = np.random.default_rng(0)
+    picks = rng.permutation(NB - 64)[:64 * 200].astype(np.int32).reshape(200, 64)
+    p.admit_into(10**6, 64 * 8, np.arange(NB - 64, NB, dtype=np.int32))     # warm-up
+    t0 = time.perf_counter()
+    for i in range(200):
+        assert p.admit_into(i, 64 * 8, picks[i]) == kvr.OK
+    per_call = (time.perf_counter() - t0) / 200
+    assert per_call < 200e-6, per_call            # ctypes marshalling included; a queue scan would cost ~1 ms
+    fq = p.free_queue()
+    named = set(picks.reshape(-1).tolist())
+    assert len(fq) == NB - 64 * 201 and not (set(fq.tolist()) & named)
+    assert fq.tolist() == [b for b in range(NB - 64) if b not in named]      # the other ids kept their order
+
+
+# ---- NUMA placement: sysfs parsing against a fake tree -------------------------------------------
+
+def test_numa_lookup_against_a_fake_sysfs_tree(tmp_path):
+    dev = tmp_path / "bus" / "pci" / "devices" / "0000:1b:00.0"
+    dev.mkdir(parents=True)
+    (dev / "numa_node").write_text("1\n")
+    node1 = tmp_path / "devices" / "system" / "node" / "node1"
+    node1.mkdir(parents=True)
+    (node1 / "cpulist").write_text("16-31,48-50,63\n")
+    node, cpus = kvr.numa_lookup(tmp_path, "0000:1B:00.0")                   # CUDA prints the bus id in upper case
+    assert node == 1 and cpus == list(range(16, 32)) + [48, 49, 50, 63]
+    # a platform that does not say (-1), a device that is not there, a malformed list
+    (dev / "numa_node").write_text("-1\n")
+    assert kvr.numa_lookup(tmp_path, "0000:1b:00.0") == (-1, [])
+    assert kvr.numa_lookup(tmp_path, "0000:ff:00.0") == (-1, [])
+    (dev / "numa_node").write_text("1\n")
+    (node1 / "cpulist").write_text("3-1\n")
+    assert kvr.numa_lookup(tmp_path, "0000:1b:00.0") == (1, [])
+    assert kvr.Pool(*GEOM, 8, 1 << 16, flags=kvr.METADATA_ONLY).numa_node == -1
