@@ -298,15 +298,19 @@ def run_longctx(args):
         ev = load_rate(load_launches) if load_launches else None
         t0 = time.perf_counter()
         assert pool.suspend_to_host(in_hbm)[0] == kvr.OK
+        t_s = time.perf_counter() - t0
         if not overlap:
             assert pool.wait() == kvr.OK
+        t1 = time.perf_counter()
         assert pool.resume_from_host(on_host)[0] == kvr.OK
+        t_r = time.perf_counter() - t1
         assert pool.wait() == kvr.OK, kvr.last_error()
         wall = time.perf_counter() - t0
         sus = max(pool.latency(r)[2] for r in in_hbm) / 1e3
         res = max(pool.latency(r)[2] for r in on_host) / 1e3
         out = {"suspend_gbs": half_bytes / sus / 1e9, "resume_gbs": half_bytes / res / 1e9,
-               "both_directions_gbs": 2 * half_bytes / wall / 1e9, "wall_s": wall}
+               "both_directions_gbs": 2 * half_bytes / wall / 1e9, "wall_s": wall,
+               "suspend_call_ms": 1e3 * t_s, "resume_call_ms": 1e3 * t_r}
         if ev:
             torch.cuda.synchronize()
             out["load_gbs"] = ev[2] / ev[0].elapsed_time(ev[1]) / 1e6

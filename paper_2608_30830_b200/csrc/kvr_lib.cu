@@ -642,14 +642,25 @@ kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> &items,
   {
     uint64_t total = 0;
     for (auto &ch : pl.chunks) total += ch.bytes;
-    const uint64_t floor_piece = align_up(total / 1024 + 1, 1 << 20);
+    const uint64_t floor_piece = align_up(total / 512 + 1, 1 << 20);
     if (piece < floor_piece) piece = floor_piece;
   }
-  auto next_cut = [&](uint64_t v) -> uint64_t {
-    if (piece >= slot) { const uint64_t G = piece / slot * slot; return (v / G + 1) * G; }
-    const uint64_t slot_end = (v / slot + 1) * slot, o = v % slot;
-    const uint64_t nx = v - o + (o / piece + 1) * piece;
-    return nx < slot_end ? nx : slot_end;
+  // next cut point after virtual position v of a chunk of n_slots slots
+  auto next_cut = [&](uint64_t v, int n_slots) -> uint64_t {
+    if (piece < 2 * slot) {                       // pieces within a slot
+      const uint64_t step = piece < slot ? piece : slot;
+      const uint64_t slot_end = (v / slot + 1) * slot, o = v % slot;
+      const uint64_t nx = v - o + (o / step + 1) * step;
+      return nx < slot_end ? nx : slot_end;
+    }
+    const uint64_t G = piece / slot * slot;       // pieces of whole slots
+    if (to_linear) {                              // ... with a cut where all slots but the last are done (early release)
+      const uint64_t early = (uint64_t)(n_slots - 1) * slot;
+      const uint64_t nx = (v / G + 1) * G;
+      return (v < early && nx > early) ? early : nx;
+    }
+    if (v < slot) return slot;                    // ... after a first copy that fits the ring's one free slot
+    return slot + ((v - slot) / G + 1) * G;
   };
   const int n_ring = ring ? (int)ring->slots.size() : 1;
   for (size_t ci = 0; ci < pl.chunks.size(); ++ci) {
@@ -698,7 +709,7 @@ kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> &items,
       for (auto &cp : ch.copies)
         for (uint64_t o = 0; o < cp.bytes;) {
           const uint64_t v = cp.vpos + o;
-          uint64_t nbytes = next_cut(v) - v;
+          uint64_t nbytes = next_cut(v, ch.n_slots) - v;
           if (nbytes > cp.bytes - o) nbytes = cp.bytes - o;
           CUP(p, cudaMemcpyAsync(p->h_arena + cp.lin_off + o, ring->base + cp.ring_off + o, nbytes, cudaMemcpyDefault, c));
           p->st.d2h_copies++; p->st.d2h_bytes += nbytes;
@@ -718,7 +729,7 @@ kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> &items,
       for (auto &cp : ch.copies)
         for (uint64_t o = 0; o < cp.bytes;) {
           const uint64_t v = cp.vpos + o;
-          uint64_t nbytes = next_cut(v) - v;
+          uint64_t nbytes = next_cut(v, ch.n_slots) - v;
           if (nbytes > cp.bytes - o) nbytes = cp.bytes - o;
           for (; looked < ch.n_slots && (uint64_t)looked * slot < v + nbytes; ++looked) {
             const Slot &sl = ring->slots[(ch.first_slot + looked) % n_ring];
