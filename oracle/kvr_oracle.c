@@ -357,6 +357,68 @@ int32_t orc_request_admit_sharing(orc_pool *p, uint64_t id, int64_t n_tokens, ui
   return ORC_OK;
 }
 
+/* Shared-prefix admission for an engine that runs its own allocator: the prefix is the donor's first n_shared
+ * blocks as above, and the caller names the private blocks (each free, named once; the other free ids keep
+ * their order).  n_shared + n_private must equal ceil(n_tokens / BS). */
+int32_t orc_request_admit_sharing_into(orc_pool *p, uint64_t id, int64_t n_tokens, uint64_t donor_id, int32_t n_shared,
+                                       const int32_t *private_blocks, int32_t n_private) {
+  if (!p || n_tokens < 0 || n_shared < 0 || n_private < 0 || (n_private > 0 && !private_blocks)) return ORC_ERR_INVALID_ARG;
+  if ((int64_t)n_shared * p->BS > n_tokens) return ORC_ERR_INVALID_ARG;
+  if ((n_tokens + p->BS - 1) / p->BS != (int64_t)n_shared + (int64_t)n_private) return ORC_ERR_INVALID_ARG;
+  orc_req *r = find_req(p, id);
+  if (r && r->state != ORC_EXPIRED) return ORC_ERR_BAD_STATE;
+  int32_t nb = n_shared + n_private;
+  int32_t *table = (int32_t *)malloc(sizeof(int32_t) * (size_t)(nb ? nb : 1));
+  if (!table) return ORC_ERR_NOMEM;
+  if (n_shared > 0) {
+    if (donor_id == id) { free(table); return ORC_ERR_INVALID_ARG; }
+    orc_req *d = find_req(p, donor_id);
+    if (!d) { free(table); return ORC_ERR_UNKNOWN_REQUEST; }
+    if (d->state == ORC_ACTIVE || d->state == ORC_RETAINED) {
+      if ((int64_t)n_shared * p->BS > d->n_tokens) { free(table); return ORC_ERR_INVALID_ARG; }
+    } else if (d->state == ORC_HOST) {
+      if (n_shared > d->n_shared) { free(table); return ORC_ERR_INVALID_ARG; }
+    } else {
+      free(table);
+      return ORC_ERR_BAD_STATE;
+    }
+    memcpy(table, d->blocks, sizeof(int32_t) * (size_t)n_shared);
+  }
+  for (int32_t i = 0; i < n_private; ++i) {
+    int found = 0;
+    for (int64_t q = 0; q < p->n_free; ++q) if (p->freeq[q] == private_blocks[i]) found = 1;
+    for (int32_t j = 0; j < i; ++j) if (private_blocks[j] == private_blocks[i]) found = 0;
+    if (!found) { free(table); return ORC_ERR_INVALID_ARG; }
+  }
+  if (!r) {
+    if (p->n_reqs == p->cap_reqs) {
+      int64_t nc = p->cap_reqs ? p->cap_reqs * 2 : 16;
+      orc_req *nr = (orc_req *)realloc(p->reqs, sizeof(orc_req) * (size_t)nc);
+      if (!nr) { free(table); return ORC_ERR_NOMEM; }
+      p->reqs = nr; p->cap_reqs = nc;
+    }
+    r = &p->reqs[p->n_reqs++];
+    memset(r, 0, sizeof(*r));
+    r->id = id;
+  }
+  for (int32_t i = 0; i < n_private; ++i)
+    for (int64_t q = 0; q < p->n_free; ++q)
+      if (p->freeq[q] == private_blocks[i]) {
+        memmove(p->freeq + q, p->freeq + q + 1, sizeof(int32_t) * (size_t)(p->n_free - q - 1));
+        p->n_free -= 1;
+        break;
+      }
+  if (n_private) memcpy(table + n_shared, private_blocks, sizeof(int32_t) * (size_t)n_private);
+  r->state = ORC_ACTIVE;
+  r->n_tokens = n_tokens;
+  r->nb = nb;
+  r->n_shared = n_shared;
+  r->image_bytes = (uint64_t)(n_tokens - (int64_t)n_shared * p->BS) * p->bpt;
+  r->blocks = table;
+  ref_blocks(p, r->blocks, nb);
+  return ORC_OK;
+}
+
 /* admission into blocks the caller names (an engine with its own allocator mirrors its choice here):
  * every block must be free and named once; the other free ids keep their order */
 int32_t orc_request_admit_into(orc_pool *p, uint64_t id, int64_t n_tokens, const int32_t *blocks, int32_t nb) {

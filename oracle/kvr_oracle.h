@@ -95,6 +95,8 @@ int32_t orc_request_admit_into(orc_pool *, uint64_t id, int64_t n_tokens, const 
  * tokens [n_shared*BS, n_tokens), (n_tokens - n_shared*BS) * bytes_per_token bytes. */
 int32_t orc_request_admit_sharing(orc_pool *, uint64_t id, int64_t n_tokens, uint64_t donor_id, int32_t n_shared,
                                   int32_t *out_blocks, int32_t cap);
+int32_t orc_request_admit_sharing_into(orc_pool *, uint64_t id, int64_t n_tokens, uint64_t donor_id, int32_t n_shared,
+                                       const int32_t *private_blocks, int32_t n_private);
 int32_t orc_request_sharing(orc_pool *, uint64_t id, int32_t *n_shared, int32_t *blocks, int32_t cap);
 int32_t orc_block_refcount(orc_pool *, int32_t blk);
 int32_t orc_request_release(orc_pool *, uint64_t id);

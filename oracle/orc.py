@@ -74,6 +74,8 @@ def lib():
         L.orc_request_release.argtypes = [vp, u64]
         L.orc_request_admit_sharing.restype = i32
         L.orc_request_admit_sharing.argtypes = [vp, u64, i64, u64, i32, pi32, i32]
+        L.orc_request_admit_sharing_into.restype = i32
+        L.orc_request_admit_sharing_into.argtypes = [vp, u64, i64, u64, i32, pi32, i32]
         L.orc_request_sharing.restype = i32
         L.orc_request_sharing.argtypes = [vp, u64, pi32, pi32, i32]
         L.orc_block_refcount.restype = i32
@@ -179,6 +181,10 @@ class OrcPool:
         out = np.zeros(max(nb, 1), dtype=np.int32)
         st = lib().orc_request_admit_sharing(self._h, rid, n_tokens, donor, n_shared, _i32p(out), nb)
         return st, (out[:nb].copy() if st == OK else None)
+
+    def admit_sharing_into(self, rid, n_tokens, donor, n_shared, private_blocks):
+        blocks = np.ascontiguousarray(private_blocks, dtype=np.int32)
+        return lib().orc_request_admit_sharing_into(self._h, rid, n_tokens, donor, n_shared, _i32p(blocks), len(blocks))
 
     def sharing(self, rid):
         """(status, shared-prefix block ids the request refers to)."""

@@ -240,3 +240,23 @@ def test_random_scripts_keep_counts_consistent(seed):
         check_counts(p, ids)
     s = p.stats()
     assert s["suspends"] > 5 and s["resumes"] + s["resident_resumes"] > 2
+
+
+def test_named_private_blocks_by_hand():
+    """An engine with its own allocator names the private blocks; the prefix still comes from the donor."""
+    p = mk(NB=10)
+    assert p.admit(1, 8)[1].tolist() == [0, 1]
+    assert p.admit_sharing_into(2, 14, 1, 2, [7, 4]) == orc.OK              # ceil(14/4) = 4 = 2 shared + 2 named
+    assert p.info(2)[1]["blocks"].tolist() == [0, 1, 7, 4] and p.sharing(2)[1].tolist() == [0, 1]
+    assert p.free_queue().tolist() == [2, 3, 5, 6, 8, 9]                    # the other free ids keep their order
+    assert [p.refcount(b) for b in (0, 1, 7, 4)] == [2, 2, 1, 1]
+    assert p.admit_sharing_into(3, 14, 1, 2, [7, 5]) == orc.ERR_INVALID_ARG     # 7 is taken
+    assert p.admit_sharing_into(3, 14, 1, 2, [5, 5]) == orc.ERR_INVALID_ARG     # named twice
+    assert p.admit_sharing_into(3, 14, 1, 2, [5]) == orc.ERR_INVALID_ARG        # 2 + 1 != 4 blocks
+    assert p.admit_sharing_into(3, 14, 9, 2, [5, 6]) == orc.ERR_UNKNOWN_REQUEST
+    assert p.admit_sharing_into(2, 14, 1, 2, [5, 6]) == orc.ERR_BAD_STATE
+    assert p.free_queue().tolist() == [2, 3, 5, 6, 8, 9]                    # failed calls changed nothing
+    assert p.suspend_to_host([2])[0] == orc.OK and p.info(2)[1]["image_bytes"] == 6 * BPT
+    assert p.free_queue().tolist() == [2, 3, 5, 6, 8, 9, 7, 4]
+    assert p.admit_sharing_into(3, 8, 2, 2, []) == orc.OK                   # everything shared, from a donor on the host
+    check_counts(p, [1, 2, 3])
