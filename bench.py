@@ -124,7 +124,7 @@ def engine_kwargs(args, kvr):
 
 
 def staging_note(args):
-    slot, n = (args.chunk_mib or 64), (args.slots or 16)
+    slot, n = (args.chunk_mib or 64), (args.slots or 32)
     return {"slot_mib": slot, "slots_per_direction": n, "staging_mib_total": 2 * slot * n,
             "largest_launch_mib": slot * (n - 1), "library_default": not (args.chunk_mib or args.slots)}
 
@@ -327,14 +327,30 @@ def run_longctx(args):
     sampler = ClockSampler(local)
     sampler.start()
     reps = max(args.steps, 1)
-    seq = median_of([exchange(False, 0) for _ in range(reps)])
-    ovl = median_of([exchange(True, 0) for _ in range(reps)])
+    peak, peak_kind = peaks()
+    keys = ("gather_launches", "scatter_launches", "gather_bytes", "scatter_bytes", "gather_ms", "scatter_ms",
+            "gather_kernel_ms", "scatter_kernel_ms")
+
+    def phase(fn):
+        """Run one phase; returns its result and the movers' roofline fractions over exactly its launches."""
+        a = pool.stats()
+        out = fn()
+        b = pool.stats()
+        d = {k: b[k] - a[k] for k in keys}
+        fr = {}
+        for side in ("gather", "scatter"):
+            fr[side] = {"frac": 2 * d[side + "_bytes"] / max(d[side + "_ms"], 1e-9) / 1e6 / peak,
+                        "in_kernel_frac": 2 * d[side + "_bytes"] / max(d[side + "_kernel_ms"], 1e-9) / 1e6 / peak,
+                        "launches": int(d[side + "_launches"]),
+                        "avg_launch_mib": d[side + "_bytes"] / max(d[side + "_launches"], 1) / 2**20}
+        return out, fr
+    seq, fr_seq = phase(lambda: median_of([exchange(False, 0) for _ in range(reps)]))
+    ovl, fr_ovl = phase(lambda: median_of([exchange(True, 0) for _ in range(reps)]))
     # size the load so that it runs for most of the overlapped exchange
     launches = max(50, int(0.8 * ovl["wall_s"] * load_alone * 1e9 / load_bytes))
-    ovl_load = median_of([exchange(True, launches) for _ in range(reps)])
+    ovl_load, fr_load = phase(lambda: median_of([exchange(True, launches) for _ in range(reps)]))
     clocks = sampler.stop()
     st = pool.stats()
-    peak, peak_kind = peaks()
     out = {
         "metric": "suspend/resume payload GB/s, both directions overlapped beside a synthetic HBM-read load",
         "value": ovl_load["both_directions_gbs"], "unit": "GB/s", "n_gpus": 1, "steps": reps, "warmup": 1,
@@ -354,6 +370,8 @@ def run_longctx(args):
             "load_loss_pct": 100 * (1 - ovl_load["load_gbs"] / load_alone)},
         "host_link": link, "clocks": clocks,
         "roofline": {"bound": "hbm", "peak": peak, "unit": "GB/s", "tile_bytes": BS * H * D * e,
+                     "by_phase": {"one_direction_at_a_time": fr_seq, "both_directions": fr_ovl,
+                                  "both_directions_beside_the_load": fr_load},
                      "gather_frac": 2 * st["gather_bytes"] / max(st["gather_ms"], 1e-9) / 1e6 / peak,
                      "scatter_frac": 2 * st["scatter_bytes"] / max(st["scatter_ms"], 1e-9) / 1e6 / peak,
                      "gather_launches": int(st["gather_launches"]), "scatter_launches": int(st["scatter_launches"]),
@@ -821,8 +839,8 @@ def main():
     ap.add_argument("--layout", default="layer", choices=["layer", "block"], help="pool layout: layer-major or block-major")
     ap.add_argument("--kernel", default="bulk", choices=["warp", "bulk"])
     ap.add_argument("--chunk-mib", type=int, default=0, help="staging slot size (0 = the library's default, 64)")
-    ap.add_argument("--slots", type=int, default=0, help="staging slots per direction (0 = the library's default, 16)")
-    ap.add_argument("--ramp-mib", type=int, default=0, help="size limit of a move's first chunk (0 = library default, 256)")
+    ap.add_argument("--slots", type=int, default=0, help="staging slots per direction (0 = the library's default, 32)")
+    ap.add_argument("--ramp-mib", type=int, default=0, help="largest move that goes in one launch (0 = library default, 1024)")
     ap.add_argument("--copy-piece-mib", type=int, default=int(os.environ.get("KVR_COPY_PIECE_MIB", "0")),
                     help="largest single link copy (0 = library default, 64)")
     ap.add_argument("--bulk-shape", default=os.environ.get("KVR_BULK_SHAPE", ""), help="bulk mover shape: warps,stages,piece_bytes")

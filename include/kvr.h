@@ -119,9 +119,11 @@ typedef struct {
   uint64_t chunk_bytes;              /* staging slot size: the granule in which staging memory is reused and the
                                         largest single copy over the link; multiple of 4096, at least one tile;
                                         0 = 64 MiB */
-  int32_t staging_slots;             /* slots per direction, in [2, 64]; 0 = 16.  Staging memory is one ring of
-                                        staging_slots x chunk_bytes per direction (default 2 x 1 GiB); one mover
-                                        launch covers up to staging_slots - 1 consecutive slots of its ring */
+  int32_t staging_slots;             /* slots per direction, in [2, 64]; 0 = 32.  Staging memory is one ring of
+                                        staging_slots x chunk_bytes per direction (default 2 x 2 GiB, 2.2 % of a
+                                        B200's memory; the link runs as fast with less, only the launches get
+                                        smaller); one mover launch covers up to staging_slots - 1 consecutive
+                                        slots of its ring */
   int32_t route;                     /* KVR_ROUTE_* */
   int32_t kernel;                    /* KVR_KERNEL_*; 0 = KVR_KERNEL_BULK */
   int32_t max_ctas;                  /* cap on the movers' grid (0 = fill the GPU) */
@@ -148,7 +150,7 @@ typedef struct {
                                         first launch of a suspend and the last launch of a resume down to one slot
                                         (so the link starts at once and little scattering remains after the last
                                         byte) and makes every other launch as large as the ring allows.
-                                        0 = 256 MiB: 85 us of mover time */
+                                        0 = 1 GiB: 0.35 ms of mover time, 2 % of such a move's time on the link */
   uint64_t copy_piece_bytes;         /* link copies are issued in pieces of at most this size (and never across a
                                         staging slot unless it is larger than a slot); 0 = 64 MiB */
   int32_t max_moves_in_flight;       /* descriptor buffers created with the pool, one per move in flight, in
@@ -232,6 +234,11 @@ kvr_status kvr_request_release(kvr_pool *pool, uint64_t req_id);
  */
 kvr_status kvr_request_admit_sharing(kvr_pool *pool, uint64_t req_id, int64_t n_tokens, uint64_t donor_id,
                                      int32_t n_shared_blocks, int32_t *out_blocks, int32_t cap);
+/* The same for an engine that runs its own allocator: the prefix comes from the donor, the private blocks are named
+ * by the caller (n_private ids, each currently free, no repeats; the other free ids keep their order);
+ * n_shared_blocks + n_private must equal ceil(n_tokens / block_size). */
+kvr_status kvr_request_admit_sharing_into(kvr_pool *pool, uint64_t req_id, int64_t n_tokens, uint64_t donor_id,
+                                          int32_t n_shared_blocks, const int32_t *private_blocks, int32_t n_private);
 /* The shared prefix a request refers to: its length in blocks and (cap entries, may be NULL) the ids. */
 kvr_status kvr_request_sharing(kvr_pool *pool, uint64_t req_id, int32_t *n_shared_blocks, int32_t *blocks, int32_t cap);
 /* Number of references to one block (0 = free); -1 for an id out of range. */

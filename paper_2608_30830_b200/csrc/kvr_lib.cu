@@ -177,7 +177,7 @@ struct kvr_pool {
   BulkShape bulk{4, 4, 8192};
   uint32_t call_flags = 0;                // flags of the call being served (set under the pool's lock)
   uint64_t copy_piece = 64ull << 20;      // largest single cudaMemcpyAsync of the staged route
-  uint64_t ramp_start = 256ull << 20;     // size limit of a move's first chunk
+  uint64_t ramp_start = 1ull << 30;       // moves up to this size are one launch (if they fit the ring)
   std::vector<cudaEvent_t> event_pool;
   std::map<uint64_t, Op> ops;
   uint64_t next_seq = 1;
@@ -349,7 +349,7 @@ struct Plan {
 // the first gather, and a resume's last scatter starts only after the last byte has arrived.  The movers are ~50
 // times faster than the link, so it is enough to keep the first chunk of a suspend and the last chunk of a resume
 // small -- one staging slot -- and let every other chunk be as large as the ring allows (`big`: all slots but one):
-//   up to ramp_start bytes (256 MiB: 85 us of mover time) a move is one launch;
+//   up to ramp_start bytes (1 GiB: 0.35 ms of mover time against 19 ms on the link) a move is one launch, if the ring holds it;
 //   suspend: [slot] [big] [big] ... [rest];      resume: [big] [big] ... [rest - slot] [slot].
 uint64_t next_cap(const kvr_pool *p, uint64_t done, uint64_t total, bool resume, uint64_t big) {
   const uint64_t tile = (uint64_t)p->tile_bytes, slot = p->slot_bytes;
@@ -1126,7 +1126,7 @@ kvr_status kvr_pool_create(const kvr_config *cfg, kvr_pool **out) {
     p->cfg.chunk_bytes = 64ull << 20;
     if (p->cfg.chunk_bytes < tile) p->cfg.chunk_bytes = align_up(tile, 4096);
   }
-  if (!p->cfg.staging_slots) p->cfg.staging_slots = 16;
+  if (!p->cfg.staging_slots) p->cfg.staging_slots = 32;
   if (!p->cfg.kernel) p->cfg.kernel = KVR_KERNEL_BULK;
   if (!p->cfg.max_moves_in_flight) p->cfg.max_moves_in_flight = 16;
   if (p->cfg.ramp_start_bytes) p->ramp_start = p->cfg.ramp_start_bytes;
@@ -1220,6 +1220,54 @@ kvr_status kvr_request_admit_sharing(kvr_pool *p, uint64_t id, int64_t n_tokens,
   }
   try {
     return admit_common(p, enter.lock, id, n_tokens, donor, n_shared, out_blocks);
+  } catch (const std::bad_alloc &) {
+    return fail(KVR_ERR_NOMEM, "out of host memory");
+  }
+}
+
+kvr_status kvr_request_admit_sharing_into(kvr_pool *p, uint64_t id, int64_t n_tokens, uint64_t donor_id, int32_t n_shared,
+                                          const int32_t *private_blocks, int32_t n_private) {
+  if (kvr_status s = check_pool(p)) return s;
+  Enter enter(p);
+  if (n_tokens < 0 || n_shared < 0 || n_private < 0 || (n_private > 0 && !private_blocks)) return fail(KVR_ERR_INVALID_ARG, "bad size or block list");
+  if ((int64_t)n_shared * p->BS > n_tokens) return fail(KVR_ERR_INVALID_ARG, "the shared prefix must be whole blocks inside the request");
+  if ((n_tokens + p->BS - 1) / p->BS != (int64_t)n_shared + (int64_t)n_private)
+    return fail(KVR_ERR_INVALID_ARG, "shared + private blocks must equal ceil(n_tokens / block_size)");
+  auto it = p->reqs.find(id);
+  if (it != p->reqs.end() && it->second.state != KVR_EXPIRED) return fail(KVR_ERR_BAD_STATE, "request exists");
+  const bool existed = it != p->reqs.end();
+  try {
+    const int32_t nb = n_shared + n_private;
+    std::vector<int32_t> table((size_t)nb), prevs((size_t)n_private);
+    if (n_shared > 0) {
+      if (donor_id == id) return fail(KVR_ERR_INVALID_ARG, "a request cannot share with itself");
+      auto d = p->reqs.find(donor_id);
+      if (d == p->reqs.end()) return fail(KVR_ERR_UNKNOWN_REQUEST, "unknown donor");
+      const Request &donor = d->second;
+      if (donor.state == KVR_ACTIVE || donor.state == KVR_RETAINED) {
+        if ((int64_t)n_shared * p->BS > donor.n_tokens) return fail(KVR_ERR_INVALID_ARG, "the donor has fewer full blocks");
+      } else if (donor.state == KVR_HOST) {
+        if (n_shared > donor.n_shared) return fail(KVR_ERR_INVALID_ARG, "a donor on the host refers only to its own shared prefix");
+      } else {
+        return fail(KVR_ERR_BAD_STATE, "a discarded donor refers to no blocks");
+      }
+      for (int32_t i = 0; i < n_shared; ++i) table[i] = donor.blocks[i];
+    }
+    Request &r = p->reqs[id];
+    uint64_t tag = 0;
+    int32_t bad = -1;
+    if (!p->fq.claim(private_blocks, n_private, prevs.data(), &tag, &bad)) {
+      if (!existed) p->reqs.erase(id);
+      return fail(KVR_ERR_INVALID_ARG, "block %d is not free or named twice", bad);
+    }
+    for (int32_t i = 0; i < n_private; ++i) table[n_shared + i] = private_blocks[i];
+    r = Request();
+    r.state = KVR_ACTIVE; r.n_tokens = n_tokens; r.nb = nb; r.n_shared = n_shared;
+    r.image_bytes = (uint64_t)(n_tokens - (int64_t)n_shared * p->BS) * p->bpt;
+    r.blocks.swap(table);
+    for (int32_t i = 0; i < n_shared; ++i) p->fq.add_ref(r.blocks[i]);
+    if (tag && !p->meta_only) return wait_unlocked(p, enter.lock, tag, true, 60000);     // a gather may still be reading the named blocks
+    return KVR_OK;
   } catch (const std::bad_alloc &) {
     return fail(KVR_ERR_NOMEM, "out of host memory");
   }

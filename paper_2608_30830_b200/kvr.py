@@ -76,7 +76,7 @@ class Stats(C.Structure):
 
 EXPORTS = [
     "kvr_bytes_per_token", "kvr_pool_create", "kvr_pool_destroy", "kvr_request_admit", "kvr_request_admit_into", "kvr_request_release",
-    "kvr_request_admit_sharing", "kvr_request_sharing", "kvr_block_refcount", "kvr_test_fail_nth", "kvr_test_points",
+    "kvr_request_admit_sharing", "kvr_request_admit_sharing_into", "kvr_request_sharing", "kvr_block_refcount", "kvr_test_fail_nth", "kvr_test_points",
     "kvr_pool_numa_node", "kvr_numa_lookup",
     "kvr_retain_in_hbm", "kvr_suspend_to_host", "kvr_expire", "kvr_resume_from_host",
     "kvr_resume_from_host_into", "kvr_export_to_device", "kvr_import_from_device", "kvr_request_info",
@@ -118,6 +118,8 @@ def lib():
     L.kvr_request_release.argtypes = [vp, u64]
     L.kvr_request_admit_sharing.restype = i32
     L.kvr_request_admit_sharing.argtypes = [vp, u64, i64, u64, i32, pi32, i32]
+    L.kvr_request_admit_sharing_into.restype = i32
+    L.kvr_request_admit_sharing_into.argtypes = [vp, u64, i64, u64, i32, pi32, i32]
     L.kvr_request_sharing.restype = i32
     L.kvr_request_sharing.argtypes = [vp, u64, pi32, pi32, i32]
     L.kvr_block_refcount.restype = i32
@@ -401,6 +403,10 @@ class Pool:
         out = np.zeros(max(nb, 1), dtype=np.int32)
         st = lib().kvr_request_admit_sharing(self._h, rid, n_tokens, donor, n_shared, _i32p(out), nb)
         return st, (out[:nb].copy() if st == OK else None)
+
+    def admit_sharing_into(self, rid, n_tokens, donor, n_shared, private_blocks):
+        blocks = np.ascontiguousarray(private_blocks, dtype=np.int32)
+        return lib().kvr_request_admit_sharing_into(self._h, rid, n_tokens, donor, n_shared, _i32p(blocks), len(blocks))
 
     def sharing(self, rid):
         """(status, shared-prefix block ids the request refers to)."""

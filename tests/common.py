@@ -18,12 +18,12 @@ def random_script(seed, n_ops, max_tokens, n_ids=12, batch=4, sharing=False):
     kinds = ["admit", "admit", "admit_into", "retain", "suspend", "suspend", "expire", "resume", "resume",
              "resume_into", "release"]
     if sharing:
-        kinds += ["admit_sharing", "admit_sharing", "admit_sharing"]
+        kinds += ["admit_sharing", "admit_sharing", "admit_sharing", "admit_sharing_into"]
     for _ in range(n_ops):
         kind = rng.choice(kinds)
-        if kind == "admit_sharing":
-            ops.append(("admit_sharing", int(rng.integers(n_ids)), int(rng.integers(0, max_tokens + 1)),
-                        int(rng.integers(n_ids)), int(rng.integers(0, 5))))
+        if kind in ("admit_sharing", "admit_sharing_into"):
+            ops.append((kind, int(rng.integers(n_ids)), int(rng.integers(0, max_tokens + 1)),
+                        int(rng.integers(n_ids)), int(rng.integers(0, 5)), int(rng.integers(2**31))))
         elif kind == "admit":
             ops.append(("admit", int(rng.integers(n_ids)), int(rng.integers(0, max_tokens + 1))))
         elif kind == "admit_into":
@@ -67,6 +67,13 @@ def run_script(pool, ops, n_ids=12, after_each=None):
         elif kind == "admit_sharing":
             st, blocks = pool.admit_sharing(op[1], op[2], op[3], op[4])
             per = None if blocks is None else blocks.tolist()
+        elif kind == "admit_sharing_into":
+            n_private = max(-(-op[2] // pool.geom[4]) - op[4], 0)
+            fq = pool.free_queue()
+            pick = np.random.default_rng(op[5]).permutation(fq)[:n_private]
+            if len(pick) < n_private:                # not enough free blocks: name an invalid list
+                pick = np.concatenate([pick, np.zeros(n_private - len(pick), dtype=np.int32) - 1])
+            st = pool.admit_sharing_into(op[1], op[2], op[3], op[4], pick.astype(np.int32))
         elif kind == "admit_into":
             bs = pool.geom[4]
             nb = -(-op[2] // bs)
