@@ -173,6 +173,7 @@ struct kvr_pool {
   Ring out_ring, in_ring;
   char *staging = nullptr; bool own_staging = false;
   uint64_t slot_bytes = 0, staging_total = 0;
+  int launch_slots = 1;                   // slots one mover launch may cover (at most all but one)
   int *status_word = nullptr;             // pinned + mapped: movers write it, the host reads it
   BulkShape bulk{4, 4, 8192};
   uint32_t call_flags = 0;                // flags of the call being served (set under the pool's lock)
@@ -372,7 +373,7 @@ uint64_t next_cap(const kvr_pool *p, uint64_t done, uint64_t total, bool resume,
 void plan_staged(kvr_pool *p, const std::vector<Item> &items, Ring &ring, bool ramp_down_too, const char *desc_dev, Plan &pl) {
   uint64_t total = 0;
   for (auto &it : items) total += (uint64_t)it.n_tokens * p->bpt;
-  const uint64_t slot = p->slot_bytes, n = ring.slots.size(), S = slot * n, big = slot * (n - 1);
+  const uint64_t slot = p->slot_bytes, n = ring.slots.size(), S = slot * n, big = slot * (uint64_t)p->launch_slots;
   int first = ring.next;
   Chunk cur;
   uint64_t vfill = 0, payload = 0, done = 0, cap = 0;
@@ -1031,6 +1032,18 @@ kvr_status create_engine(kvr_pool *p) {
     if (p->staging) {
       p->route = KVR_ROUTE_STAGED;
       p->slot_bytes = c.chunk_bytes;
+      // How many of the ring's n slots one launch may cover.  While the link drains (or fills) the slots a launch
+      // leaves free, the next launch has to run: with m slots per launch, (n - m) slots of link time must cover the
+      // mover's time for m slots.  At full speed the movers are ~50 times faster than a PCIe Gen5 link (3 TB/s of
+      // payload against 57 GB/s), which allows all slots but one; a grid capped with max_ctas is slower in
+      // proportion (bulk mover: ~20 GB/s per CTA; warp mover: ~4 GB/s per CTA), and an arena in device memory is
+      // a faster "link".  A margin of 1.5 covers launch latencies.
+      const int full_grid = c.kernel == KVR_KERNEL_BULK ? p->sm_count : 5 * p->sm_count;
+      const int grid = (c.max_ctas > 0 && c.max_ctas < full_grid) ? c.max_ctas : full_grid;
+      const double mover_gbs = 3000.0 * grid / full_grid;
+      const double link_gbs = p->arena_on_device ? 800.0 : 57.0;
+      int m = (int)((double)n * mover_gbs / (mover_gbs + 1.5 * link_gbs));
+      p->launch_slots = m < 1 ? 1 : (m > n - 1 ? n - 1 : m);
       for (int dir = 0; dir < 2; ++dir) {
         Ring &r = dir ? p->in_ring : p->out_ring;
         r.base = p->staging + (size_t)dir * n * c.chunk_bytes;
