@@ -799,7 +799,6 @@ kvr_status enqueue(kvr_pool *p, int kind, std::vector<Item> &items, int route, c
   op.kind = kind;
   kvr_status s;
   try {
-    // the event pool takes back every event of the move, whatever happens: make room now
     s = enqueue_impl(p, op, kind, items, route, lin_dev, block_tag, arena_waits, t_call, lease, out_seq);
   } catch (const std::bad_alloc &) {
     s = fail(KVR_ERR_NOMEM, "out of host memory while enqueueing a move");
@@ -1089,6 +1088,24 @@ struct Batch {
   void put(kvr_status s) { if (per) per[i] = s; acc = fold(acc, s); ++i; }
 };
 
+// Who may donate its first n_shared blocks as a shared prefix: a request that still refers to them -- ACTIVE or
+// RETAINED with that many full blocks, or on the HOST with a kept prefix at least that long.
+kvr_status check_donor(kvr_pool *p, uint64_t id, uint64_t donor_id, int32_t n_shared, const Request **out) {
+  if (donor_id == id) return fail(KVR_ERR_INVALID_ARG, "a request cannot share with itself");
+  auto d = p->reqs.find(donor_id);
+  if (d == p->reqs.end()) return fail(KVR_ERR_UNKNOWN_REQUEST, "unknown donor");
+  const Request &donor = d->second;
+  if (donor.state == KVR_ACTIVE || donor.state == KVR_RETAINED) {
+    if ((int64_t)n_shared * p->BS > donor.n_tokens) return fail(KVR_ERR_INVALID_ARG, "the donor has fewer full blocks");
+  } else if (donor.state == KVR_HOST) {
+    if (n_shared > donor.n_shared) return fail(KVR_ERR_INVALID_ARG, "a donor on the host refers only to its own shared prefix");
+  } else {
+    return fail(KVR_ERR_BAD_STATE, "a discarded donor refers to no blocks");
+  }
+  *out = &donor;
+  return KVR_OK;
+}
+
 // the new request's table: donor prefix (one more reference each) followed by ids from the head of the queue
 kvr_status admit_common(kvr_pool *p, std::unique_lock<std::mutex> &lock, uint64_t id, int64_t n_tokens, const Request *donor,
                         int32_t n_shared, int32_t *out_blocks) {
@@ -1218,19 +1235,7 @@ kvr_status kvr_request_admit_sharing(kvr_pool *p, uint64_t id, int64_t n_tokens,
   auto it = p->reqs.find(id);
   if (it != p->reqs.end() && it->second.state != KVR_EXPIRED) return fail(KVR_ERR_BAD_STATE, "request exists");
   const Request *donor = nullptr;
-  if (n_shared > 0) {
-    if (donor_id == id) return fail(KVR_ERR_INVALID_ARG, "a request cannot share with itself");
-    auto d = p->reqs.find(donor_id);
-    if (d == p->reqs.end()) return fail(KVR_ERR_UNKNOWN_REQUEST, "unknown donor");
-    donor = &d->second;
-    if (donor->state == KVR_ACTIVE || donor->state == KVR_RETAINED) {
-      if ((int64_t)n_shared * p->BS > donor->n_tokens) return fail(KVR_ERR_INVALID_ARG, "the donor has fewer full blocks");
-    } else if (donor->state == KVR_HOST) {
-      if (n_shared > donor->n_shared) return fail(KVR_ERR_INVALID_ARG, "a donor on the host refers only to its own shared prefix");
-    } else {
-      return fail(KVR_ERR_BAD_STATE, "a discarded donor refers to no blocks");
-    }
-  }
+  if (n_shared > 0) { if (kvr_status s = check_donor(p, id, donor_id, n_shared, &donor)) return s; }
   try {
     return admit_common(p, enter.lock, id, n_tokens, donor, n_shared, out_blocks);
   } catch (const std::bad_alloc &) {
@@ -1253,18 +1258,9 @@ kvr_status kvr_request_admit_sharing_into(kvr_pool *p, uint64_t id, int64_t n_to
     const int32_t nb = n_shared + n_private;
     std::vector<int32_t> table((size_t)nb), prevs((size_t)n_private);
     if (n_shared > 0) {
-      if (donor_id == id) return fail(KVR_ERR_INVALID_ARG, "a request cannot share with itself");
-      auto d = p->reqs.find(donor_id);
-      if (d == p->reqs.end()) return fail(KVR_ERR_UNKNOWN_REQUEST, "unknown donor");
-      const Request &donor = d->second;
-      if (donor.state == KVR_ACTIVE || donor.state == KVR_RETAINED) {
-        if ((int64_t)n_shared * p->BS > donor.n_tokens) return fail(KVR_ERR_INVALID_ARG, "the donor has fewer full blocks");
-      } else if (donor.state == KVR_HOST) {
-        if (n_shared > donor.n_shared) return fail(KVR_ERR_INVALID_ARG, "a donor on the host refers only to its own shared prefix");
-      } else {
-        return fail(KVR_ERR_BAD_STATE, "a discarded donor refers to no blocks");
-      }
-      for (int32_t i = 0; i < n_shared; ++i) table[i] = donor.blocks[i];
+      const Request *donor = nullptr;
+      if (kvr_status s = check_donor(p, id, donor_id, n_shared, &donor)) return s;
+      for (int32_t i = 0; i < n_shared; ++i) table[i] = donor->blocks[i];
     }
     Request &r = p->reqs[id];
     uint64_t tag = 0;

@@ -123,11 +123,12 @@ class Rig:
         """Planes [p0, p1) of the image of a request with this table and n tokens, from the pool as it is now."""
         return image_by_definition(self.dev, self.geom, self.NB, table, n, p0, p1)
 
-    def assert_whole_images(self, ids, tables, images, slab_bytes=1 << 30):
-        """Every byte of every image (numpy views of the pinned arena) against the definition under `tables`."""
+    def assert_whole_images(self, ids, tables, images, slab_bytes=1 << 30, tokens=None):
+        """Every byte of every image (numpy views of the pinned arena) against the definition under `tables`
+        (`tokens`: how many tokens each table covers, when that is not the whole request)."""
         L, H, D, e, BS = self.geom
         for rid in ids:
-            n = int(self.o.info(rid)[1]["n_tokens"])
+            n = int(tokens[rid]) if tokens is not None else int(self.o.info(rid)[1]["n_tokens"])
             if n == 0:
                 continue
             img = torch.from_numpy(images[rid]).view(2 * L, n, self.row)
@@ -367,4 +368,69 @@ def test_config5_long_context_overlapped_suspend_and_resume():
     assert bool((same | touched_mask(rig, ids).unsqueeze(0)).all())
     del same, sums0
     check_invariants(rig.g, ids)
+    rig.close()
+
+
+def test_paper_shaped_contexts_sharing_one_prefix_full_size():
+    """One TP4 rank of the paper's model (80 layers, 2 KV heads: 8 KiB tiles), 32 gate contexts of 8,400 tokens over
+    one shared 5,392-token prefix (337 whole blocks), pool at 50 % occupancy.  Only the 3,008-token suffixes move:
+    every image byte against the definition over the private part of the table, the prefix blocks untouched and
+    still referenced while the requests are on the host, every other pool row unchanged by the round trip."""
+    w = CONFIGS["paper_shape"]
+    seed = SEED + 6
+    L, H, D, e, BS = w.geom
+    bpt = kvr.bytes_per_token(*w.geom[:4])
+    n_ctx, shared_blocks = 8400, w.extra["shared_tokens"] // BS
+    n_priv = n_ctx - shared_blocks * BS
+    ids = list(range(w.n_requests))
+    host_cap = len(ids) * (n_priv * bpt + 4096) + (64 << 20)
+    rig = Rig(w.geom, w.num_blocks, host_cap, seed)
+    PREFIX = 900
+    assert rig.both("admit", PREFIX, shared_blocks * BS)[0] == kvr.OK
+    used = shared_blocks + len(ids) * (-(-n_ctx // BS) - shared_blocks)
+    fillers = occupancy_fillers(w.num_blocks, BS, used, w.occupancy, seed)
+    order = [(i, n_ctx) for i in ids] + [(1000 + i, int(n)) for i, n in enumerate(fillers)]
+    np.random.default_rng(seed).shuffle(order)
+    for rid, n in order:
+        if rid < 900:
+            a = rig.o.admit_sharing(rid, n, PREFIX, shared_blocks)
+            b = rig.g.admit_sharing(rid, n, PREFIX, shared_blocks)
+            assert a[0] == b[0] == kvr.OK and a[1].tolist() == b[1].tolist()
+        else:
+            assert rig.both("admit", rid, n)[0] == kvr.OK
+    assert rig.both("release", PREFIX) == kvr.OK
+    prefix = rig.g.sharing(0)[1]
+    assert len(prefix) == shared_blocks and rig.g.refcount(int(prefix[0])) == len(ids)
+    sums0 = rig.row_sums()
+    private = {rid: rig.o.info(rid)[1]["blocks"][shared_blocks:].copy() for rid in ids}
+    st, per = rig.both("suspend_to_host", ids)
+    assert st == kvr.OK
+    assert rig.g.wait() == kvr.OK, kvr.last_error()
+    s = rig.g.stats()
+    assert s["bytes_suspended"] == s["gather_bytes"] == len(ids) * n_priv * bpt          # 246 MB per context, not 688 MB
+    assert s["blocks_pinned"] == shared_blocks and rig.g.refcount(int(prefix[0])) == len(ids)
+    assert torch.equal(rig.row_sums(), sums0)
+    images = {rid: rig.g.host_image(rid) for rid in ids}
+    tokens = {rid: n_priv for rid in ids}
+    rig.assert_whole_images(ids, private, images, tokens=tokens)
+    ro = rig.o.resume_from_host(ids[::-1])
+    rg = rig.g.resume_from_host(ids[::-1])
+    assert ro == rg and rg[0] == kvr.OK
+    assert rig.g.wait() == kvr.OK, kvr.last_error()
+    new_private = {}
+    for rid in ids:
+        t = rig.o.info(rid)[1]["blocks"]
+        assert t.tolist() == rig.g.info(rid)[1]["blocks"].tolist() and t[:shared_blocks].tolist() == prefix.tolist()
+        new_private[rid] = t[shared_blocks:].copy()
+    rig.assert_whole_images(ids, new_private, images, tokens=tokens)
+    # nothing but the valid slots of the new private blocks changed: the shared prefix in particular did not
+    mask = torch.zeros(rig.NB, BS, dtype=torch.bool)
+    for rid in ids:
+        mask[torch.from_numpy(new_private[rid][:n_priv // BS].astype(np.int64))] = True
+        if n_priv % BS:
+            mask[int(new_private[rid][-1]), :n_priv % BS] = True
+    same = rig.row_sums() == sums0
+    assert bool((same | mask.cuda().unsqueeze(0)).all())
+    assert rig.o.free_queue().tolist() == rig.g.free_queue().tolist()
+    check_invariants(rig.g, ids + [1000 + i for i in range(len(fillers))])
     rig.close()

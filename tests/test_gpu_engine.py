@@ -96,7 +96,8 @@ def test_shared_prefix_round_trip_moves_the_suffix_only():
     geom = (4, 8, 128, 2, 16)
     bpt = kvr.bytes_per_token(*geom[:4])
     t = Twin(geom, 512, 64 << 20, seed=9)
-    assert t.both("admit", 0, 1600)[0][0] == orc.OK                          # the prefix: 100 full blocks
+    a, b = t.both("admit", 0, 1600)                                          # the prefix: 100 full blocks
+    assert a[0] == b[0] == orc.OK and a[1].tolist() == b[1].tolist()
     for rid, n in ((1, 1600 + 900), (2, 1600 + 37), (3, 1600)):
         a, b = t.both("admit_sharing", rid, n, 0, 100)
         assert a[0] == b[0] == orc.OK and a[1].tolist() == b[1].tolist()
@@ -191,7 +192,8 @@ def test_caller_owned_staging_and_streams():
              streams=[s.cuda_stream for s in streams])
     ids = list(range(6))
     for rid, n in zip(ids, (700, 33, 1, 512, 250, 90)):
-        assert t.both("admit", rid, n)[0][0] == orc.OK
+        a, b = t.both("admit", rid, n)
+        assert a[0] == b[0] == orc.OK and a[1].tolist() == b[1].tolist()
     a, b = t.both("suspend_to_host", ids)
     assert a == b
     t.assert_same_images(ids)
@@ -217,7 +219,8 @@ def test_more_moves_in_flight_than_descriptor_buffers():
     t = Twin(geom, 2048, 256 << 20, seed=3, max_moves_in_flight=2, chunk_bytes=4 << 20, staging_slots=4)
     ids = list(range(10))
     for rid in ids:
-        assert t.both("admit", rid, 1500 + 37 * rid)[0][0] == orc.OK
+        a, b = t.both("admit", rid, 1500 + 37 * rid)
+        assert a[0] == b[0] == orc.OK and a[1].tolist() == b[1].tolist()
     for rid in ids:                                                          # ten moves, no waits in between
         assert t.both("suspend_to_host", [rid]) == ((orc.OK, [orc.OK]), (kvr.OK, [kvr.OK]))
     t.assert_same_images(ids)
