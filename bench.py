@@ -117,7 +117,8 @@ def engine_kwargs(args, kvr):
     """Engine settings from the command line; 0 / unset leaves the library's own default in place."""
     kw = dict(chunk_bytes=args.chunk_mib << 20, staging_slots=args.slots, max_ctas=args.max_ctas,
               kernel={"warp": kvr.KERNEL_WARP, "bulk": kvr.KERNEL_BULK}[args.kernel],
-              ramp_start_bytes=args.ramp_mib << 20, copy_piece_bytes=args.copy_piece_mib << 20)
+              suspend_single_bytes=args.suspend_single_mib << 20, resume_single_bytes=args.resume_single_mib << 20,
+              copy_piece_bytes=args.copy_piece_mib << 20)
     if args.bulk_shape:
         kw["bulk_shape"] = tuple(int(x) for x in args.bulk_shape.split(","))
     return kw
@@ -840,7 +841,8 @@ def main():
     ap.add_argument("--kernel", default="bulk", choices=["warp", "bulk"])
     ap.add_argument("--chunk-mib", type=int, default=0, help="staging slot size (0 = the library's default, 64)")
     ap.add_argument("--slots", type=int, default=0, help="staging slots per direction (0 = the library's default, 32)")
-    ap.add_argument("--ramp-mib", type=int, default=0, help="largest move that goes in one launch (0 = library default, 1024)")
+    ap.add_argument("--suspend-single-mib", type=int, default=0, help="largest suspend that goes in one launch (0 = library default, 1024)")
+    ap.add_argument("--resume-single-mib", type=int, default=0, help="largest resume that goes in one launch (0 = library default, 256)")
     ap.add_argument("--copy-piece-mib", type=int, default=int(os.environ.get("KVR_COPY_PIECE_MIB", "0")),
                     help="largest single link copy (0 = library default, 64)")
     ap.add_argument("--bulk-shape", default=os.environ.get("KVR_BULK_SHAPE", ""), help="bulk mover shape: warps,stages,piece_bytes")

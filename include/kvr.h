@@ -146,11 +146,14 @@ typedef struct {
                                         streams of cfg->device, or NULL each: the library creates high-priority
                                         non-blocking streams.  Caller-owned streams must not be used for anything
                                         that waits on this pool's moves from inside the same stream */
-  uint64_t ramp_start_bytes;         /* a move of up to this many bytes is one mover launch; a larger one keeps the
-                                        first launch of a suspend and the last launch of a resume down to one slot
-                                        (so the link starts at once and little scattering remains after the last
-                                        byte) and makes every other launch as large as the ring allows.
-                                        0 = 1 GiB: 0.35 ms of mover time, 2 % of such a move's time on the link */
+  uint64_t suspend_single_bytes;     /* a suspend of up to this many bytes is one mover launch; a larger one keeps
+                                        its first launch down to one slot, so the link starts at once, and makes
+                                        every other launch as large as the ring allows.  0 = 1 GiB: the blocks of
+                                        such a request are free 0.35 ms later than they could be, 2 % of the
+                                        19 ms the move spends on the link */
+  uint64_t resume_single_bytes;      /* the same for a resume, whose last launch is the one kept down to a slot, so
+                                        that little scattering remains after the last byte has arrived.  0 =
+                                        256 MiB: at most 85 us between the last byte and the request being usable */
   uint64_t copy_piece_bytes;         /* link copies are issued in pieces of at most this size (and never across a
                                         staging slot unless it is larger than a slot); 0 = 64 MiB */
   int32_t max_moves_in_flight;       /* descriptor buffers created with the pool, one per move in flight, in

@@ -178,7 +178,8 @@ struct kvr_pool {
   BulkShape bulk{4, 4, 8192};
   uint32_t call_flags = 0;                // flags of the call being served (set under the pool's lock)
   uint64_t copy_piece = 64ull << 20;      // largest single cudaMemcpyAsync of the staged route
-  uint64_t ramp_start = 1ull << 30;       // moves up to this size are one launch (if they fit the ring)
+  uint64_t suspend_single = 1ull << 30;   // a suspend up to this size is one launch (if it fits the ring)
+  uint64_t resume_single = 256ull << 20;  // a resume up to this size is one launch
   std::vector<cudaEvent_t> event_pool;
   std::map<uint64_t, Op> ops;
   uint64_t next_seq = 1;
@@ -349,14 +350,16 @@ struct Plan {
 // launches; what speaks against one single launch is latency at the link: a suspend's first byte crosses only after
 // the first gather, and a resume's last scatter starts only after the last byte has arrived.  The movers are ~50
 // times faster than the link, so it is enough to keep the first chunk of a suspend and the last chunk of a resume
-// small -- one staging slot -- and let every other chunk be as large as the ring allows (`big`: all slots but one):
-//   up to ramp_start bytes (1 GiB: 0.35 ms of mover time against 19 ms on the link) a move is one launch, if the ring holds it;
+// small -- one staging slot -- and let every other chunk be as large as the ring allows (`big`):
 //   suspend: [slot] [big] [big] ... [rest];      resume: [big] [big] ... [rest - slot] [slot].
+// Below a size threshold the split is not worth a launch and the move goes in one: 1 GiB for a suspend (its blocks
+// are free 0.35 ms later, 2 % of the move), 256 MiB for a resume (at most 85 us between the last byte and a usable
+// request: a resume's latency is what the caller waits for).
 uint64_t next_cap(const kvr_pool *p, uint64_t done, uint64_t total, bool resume, uint64_t big) {
   const uint64_t tile = (uint64_t)p->tile_bytes, slot = p->slot_bytes;
   const uint64_t left = total > done ? total - done : 0;
   uint64_t cap = big;
-  if (total > p->ramp_start && total > 2 * slot) {
+  if (total > (resume ? p->resume_single : p->suspend_single) && total > 2 * slot) {
     if (!resume) { if (done == 0) cap = slot; }
     else if (left > 2 * slot && left <= big + slot) cap = left - slot;
   }
@@ -1036,12 +1039,14 @@ kvr_status create_engine(kvr_pool *p) {
       // mover's time for m slots.  At full speed the movers are ~50 times faster than a PCIe Gen5 link (3 TB/s of
       // payload against 57 GB/s), which allows all slots but one; a grid capped with max_ctas is slower in
       // proportion (bulk mover: ~20 GB/s per CTA; warp mover: ~4 GB/s per CTA), and an arena in device memory is
-      // a faster "link".  A margin of 1.5 covers launch latencies.
+      // a faster "link".  A margin of 1.5 covers launch latencies; a capped grid never takes more than half the ring
+      // (whoever capped it runs other kernels beside the movers, which may slow them further).
       const int full_grid = c.kernel == KVR_KERNEL_BULK ? p->sm_count : 5 * p->sm_count;
       const int grid = (c.max_ctas > 0 && c.max_ctas < full_grid) ? c.max_ctas : full_grid;
       const double mover_gbs = 3000.0 * grid / full_grid;
       const double link_gbs = p->arena_on_device ? 800.0 : 57.0;
       int m = (int)((double)n * mover_gbs / (mover_gbs + 1.5 * link_gbs));
+      if (grid < full_grid && m > n / 2) m = n / 2;     // a capped grid shares the SMs with somebody: plain double buffering
       p->launch_slots = m < 1 ? 1 : (m > n - 1 ? n - 1 : m);
       for (int dir = 0; dir < 2; ++dir) {
         Ring &r = dir ? p->in_ring : p->out_ring;
@@ -1159,7 +1164,8 @@ kvr_status kvr_pool_create(const kvr_config *cfg, kvr_pool **out) {
   if (!p->cfg.staging_slots) p->cfg.staging_slots = 32;
   if (!p->cfg.kernel) p->cfg.kernel = KVR_KERNEL_BULK;
   if (!p->cfg.max_moves_in_flight) p->cfg.max_moves_in_flight = 16;
-  if (p->cfg.ramp_start_bytes) p->ramp_start = p->cfg.ramp_start_bytes;
+  if (p->cfg.suspend_single_bytes) p->suspend_single = p->cfg.suspend_single_bytes;
+  if (p->cfg.resume_single_bytes) p->resume_single = p->cfg.resume_single_bytes;
   if (p->cfg.copy_piece_bytes) p->copy_piece = p->cfg.copy_piece_bytes;
   kvr_status bad = KVR_OK;
   if (p->cfg.route < KVR_ROUTE_AUTO || p->cfg.route > KVR_ROUTE_DMA2D) bad = fail(KVR_ERR_INVALID_ARG, "unknown route");

@@ -38,7 +38,7 @@ class Config(C.Structure):
                 ("device_pool", C.c_void_p), ("host_arena", C.c_void_p),
                 ("initial_free_order", C.POINTER(C.c_int32)),
                 ("device_staging", C.c_void_p), ("streams", C.c_void_p * 4),
-                ("ramp_start_bytes", C.c_uint64), ("copy_piece_bytes", C.c_uint64),
+                ("suspend_single_bytes", C.c_uint64), ("resume_single_bytes", C.c_uint64), ("copy_piece_bytes", C.c_uint64),
                 ("max_moves_in_flight", C.c_int32), ("bulk_warps", C.c_int32), ("bulk_stages", C.c_int32),
                 ("bulk_piece_bytes", C.c_int32)]
 
@@ -333,7 +333,8 @@ class Pool:
     def __init__(self, layers, kv_heads, head_dim, dtype_bytes, block_size, num_blocks, host_capacity_bytes,
                  initial_free_order=None, device=0, chunk_bytes=0, staging_slots=0, route=0, kernel=0,
                  max_ctas=0, flags=0, device_pool=None, host_arena=None, layout=0, device_staging=None, streams=None,
-                 ramp_start_bytes=0, copy_piece_bytes=0, max_moves_in_flight=0, bulk_shape=None):
+                 suspend_single_bytes=0, resume_single_bytes=0, copy_piece_bytes=0, max_moves_in_flight=0,
+                 bulk_shape=None):
         self.geom = (layers, kv_heads, head_dim, dtype_bytes, block_size)
         self.NB = num_blocks
         cfg = Config()
@@ -350,7 +351,8 @@ class Pool:
                 raise ValueError("streams: gather, d2h, h2d, scatter")
             for i, st in enumerate(streams):
                 cfg.streams[i] = st
-        cfg.ramp_start_bytes, cfg.copy_piece_bytes, cfg.max_moves_in_flight = ramp_start_bytes, copy_piece_bytes, max_moves_in_flight
+        cfg.suspend_single_bytes, cfg.resume_single_bytes = suspend_single_bytes, resume_single_bytes
+        cfg.copy_piece_bytes, cfg.max_moves_in_flight = copy_piece_bytes, max_moves_in_flight
         if bulk_shape is not None:
             cfg.bulk_warps, cfg.bulk_stages, cfg.bulk_piece_bytes = bulk_shape
         order = None

@@ -184,3 +184,47 @@ def test_controller_rejects_bad_configs_and_time_travel():
     assert c.suspend(1, 100.0) == kvr.OK
     assert c.advance(50.0)[0] == kvr.ERR_INVALID_ARG                   # the clock never runs backwards
     assert c.suspend(1, 101.0) == kvr.ERR_BAD_STATE and c.resume(7, 102.0) == kvr.ERR_UNKNOWN_REQUEST
+
+
+class SharingPool:
+    """A pool whose plain admissions share the first `ns` blocks of a long-lived donor request: the paper's workload
+    shape (one system prefix, private suffixes) driven through code that only knows `admit`."""
+
+    def __init__(self, pool, donor, ns, bs):
+        self._pool, self._donor, self._ns, self._bs = pool, donor, ns, bs
+
+    def admit(self, rid, n_private):
+        return self._pool.admit_sharing(rid, self._ns * self._bs + n_private, self._donor, self._ns)
+
+    def __getattr__(self, name):
+        return getattr(self._pool, name)
+
+
+def test_library_controller_matches_the_oracle_over_a_shared_prefix():
+    """Every context shares one system prefix (Section 2): the tier holds private suffixes only, the prefix stays
+    resident while any context refers to it, and the library's controller decides exactly as the oracle's."""
+    n, NB, host_cap, ns, PREFIX = 160, 700, 32 * 4096, 9, 10_000
+    rng = np.random.default_rng(41)
+    lengths = rng.integers(1, 100, size=n)
+    mean_img = float(np.mean(lengths)) * 64
+    w_ref = 1800.0
+    lam = 2.5 * (host_cap / mean_img) / w_ref
+    arrive, wait = poisson_arrivals(n, lam, 41), paper_wait_family("mixture", n, 41)
+    order = rng.permutation(NB).astype(np.int32)
+    po = orc.OrcPool(*GEOM, NB, host_cap, initial_free_order=order, with_data=False)
+    pg = kvr.Pool(*GEOM, NB, host_cap, initial_free_order=order, flags=kvr.METADATA_ONLY)
+    for pool in (po, pg):
+        assert pool.admit(PREFIX, ns * 4)[0] == orc.OK
+    co = OrcController(po, PRICES, lam, w_ref, mean_image_bytes=mean_img, hbm_grace_s=20.0, branch=TTL, admission=LIVE)
+    cg = kvr.Controller(pg, PRICES, lam, w_ref, mean_image_bytes=mean_img, hbm_grace_s=20.0, branch=TTL, admission=LIVE)
+    lo = run_trace(co, SharingPool(po, PREFIX, ns, 4), arrive, wait, lengths)
+    lg = run_trace(cg, SharingPool(pg, PREFIX, ns, 4), arrive, wait, lengths)
+    assert lo == lg
+    so, sg = co.stats(), cg.stats()
+    for k in so:
+        assert sg[k] == pytest.approx(so[k], rel=1e-12), k
+    ids = list(range(n)) + [PREFIX]
+    assert snapshot(po, ids) == snapshot(pg, ids)
+    assert so["resumed_host"] > 10 and so["offloaded"] > 50
+    assert po.stats()["bytes_suspended"] == pg.stats()["bytes_suspended"] < so["offloaded"] * 100 * 64     # suffixes only
+    assert pg.refcount(int(pg.info(PREFIX)[1]["blocks"][0])) == 1            # every sharer has let go again

@@ -18,8 +18,8 @@ SMALL = (3, 2, 16, 2, 8)          # L, H, D, e, BS: 64-byte rows, 512-byte tiles
 
 RINGS = [
     pytest.param(dict(chunk_bytes=4096, staging_slots=3), id="3x4K"),
-    pytest.param(dict(chunk_bytes=4096, staging_slots=5, ramp_start_bytes=8192), id="5x4K-ramp8K"),
-    pytest.param(dict(chunk_bytes=8192, staging_slots=16, ramp_start_bytes=4096, copy_piece_bytes=4096), id="16x8K-piece4K"),
+    pytest.param(dict(chunk_bytes=4096, staging_slots=5, suspend_single_bytes=8192, resume_single_bytes=8192), id="5x4K-single8K"),
+    pytest.param(dict(chunk_bytes=8192, staging_slots=16, suspend_single_bytes=4096, resume_single_bytes=4096, copy_piece_bytes=4096), id="16x8K-piece4K"),
     pytest.param(dict(chunk_bytes=4096, staging_slots=7, copy_piece_bytes=12288), id="7x4K-piece12K"),
     pytest.param(dict(chunk_bytes=12288, staging_slots=4, kernel=kvr.KERNEL_WARP), id="4x12K-warp"),
 ]
@@ -48,7 +48,7 @@ def test_one_large_batch_through_a_small_ring():
     """One batched suspend and resume of 40 ragged requests through a 6-slot ring: launches of up to five slots,
     dozens of wraps, every image and the whole pool against the oracle."""
     geom = (2, 8, 128, 2, 16)                     # 2 KiB rows, 32 KiB tiles, 8 KiB per token
-    t = Twin(geom, 2048, 160 << 20, seed=4, chunk_bytes=1 << 20, staging_slots=6, ramp_start_bytes=2 << 20)
+    t = Twin(geom, 2048, 160 << 20, seed=4, chunk_bytes=1 << 20, staging_slots=6, suspend_single_bytes=2 << 20, resume_single_bytes=2 << 20)
     rng = np.random.default_rng(4)
     lens = [int(x) for x in rng.integers(1, 700, size=40)]
     ids = list(range(40))

@@ -171,3 +171,75 @@ def test_live_controller_with_data():
     t.assert_same_pool()
     cg.close()
     t.close()
+
+
+class _SharingPool:
+    """A pool whose plain admissions share the first `ns` blocks of a long-lived donor request: the paper's workload
+    shape (one system prefix, private suffixes) driven through code that only knows `admit`."""
+
+    def __init__(self, pool, donor, ns, bs):
+        self._pool, self._donor, self._ns, self._bs = pool, donor, ns, bs
+
+    def admit(self, rid, n_private):
+        return self._pool.admit_sharing(rid, self._ns * self._bs + n_private, self._donor, self._ns)
+
+    def __getattr__(self, name):
+        return getattr(self._pool, name)
+
+
+def test_live_controller_over_a_shared_prefix_with_data():
+    """The live controller when every context shares one system prefix: only private suffixes travel, the prefix
+    stays resident as long as any context (active, pinned or on the host) refers to it, and decisions, costs, images
+    and final pool bytes equal the oracle's."""
+    from kvr_synth import paper_wait_family, poisson_arrivals
+    from oracle.controller import LIVE, TTL, OrcController
+    from test_controller_cpu import PRICES, run_trace
+    geom = (2, 2, 16, 2, 4)                        # 256 bytes per token
+    L, H, D, e, BS = geom
+    n, NB, host_cap, ns = 160, 700, 32 * 4096, 9   # a 36-token prefix
+    rng = np.random.default_rng(41)
+    lengths = rng.integers(1, 100, size=n)         # private suffix lengths
+    mean_img = float(np.mean(lengths)) * 256
+    w_ref = 1800.0
+    lam = 2.5 * (host_cap / mean_img) / w_ref
+    arrive, wait = poisson_arrivals(n, lam, 41), paper_wait_family("mixture", n, 41)
+    t = Twin(geom, NB, host_cap, seed=41, chunk_bytes=8192, staging_slots=3)
+    o_view = t.o.data.reshape(2 * L, NB, BS * H * D * e)
+    d_view = t.dev.view(2 * L, NB, BS * H * D * e)
+    PREFIX = 10_000
+    a, b = t.both("admit", PREFIX, ns * BS)
+    assert a[0] == b[0] == orc.OK and a[1].tolist() == b[1].tolist()
+    prefix_blocks = a[1]
+    fills = {}
+    pool_is_gpu = [False]
+
+    def on_admit(i, blocks):                       # fresh bytes for the private blocks only, the same on both sides
+        assert blocks[:ns].tolist() == prefix_blocks.tolist()
+        mine = blocks[ns:]
+        k = fills.get(i, 0)
+        fills[i] = k + 1
+        fresh = np.random.default_rng([41, i, k]).integers(0, 256, size=(2 * L, len(mine), BS * H * D * e), dtype=np.uint8)
+        if pool_is_gpu[0]:
+            d_view[:, torch.from_numpy(mine.astype(np.int64)).cuda()] = torch.from_numpy(fresh).cuda()
+            torch.cuda.synchronize()
+        else:
+            o_view[:, mine] = fresh
+    so_pool, sg_pool = _SharingPool(t.o, PREFIX, ns, BS), _SharingPool(t.g, PREFIX, ns, BS)
+    co = OrcController(t.o, PRICES, lam, w_ref, mean_image_bytes=mean_img, hbm_grace_s=20.0, branch=TTL, admission=LIVE)
+    lo = run_trace(co, so_pool, arrive, wait, lengths, on_admit=on_admit)
+    pool_is_gpu[0] = True
+    fills.clear()
+    cg = kvr.Controller(t.g, PRICES, lam, w_ref, mean_image_bytes=mean_img, hbm_grace_s=20.0, branch=TTL, admission=kvr.ADMIT_LIVE)
+    lg = run_trace(cg, sg_pool, arrive, wait, lengths, on_admit=on_admit)
+    assert lo == lg
+    so, sg = co.stats(), cg.stats()
+    for k in so:
+        assert sg[k] == pytest.approx(so[k], rel=1e-12), k
+    assert so["resumed_host"] > 15 and so["ttl_expired"] + so["evicted_lru"] > 0
+    ps, pg = t.o.stats(), t.g.stats()
+    assert ps["bytes_suspended"] == pg["bytes_suspended"] == pg["gather_bytes"] > 0      # suffix bytes only
+    assert t.g.refcount(int(prefix_blocks[0])) == t.o.refcount(int(prefix_blocks[0])) == 1     # only the owner is left
+    t.assert_same_pool()
+    check_invariants(t.g, list(range(n)) + [PREFIX])
+    cg.close()
+    t.close()
