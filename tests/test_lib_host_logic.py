@@ -224,9 +224,10 @@ def test_paper_context_split_in_the_library(golden):
     983,040,000 bytes (0.98 GB), not 2.75 GB; the prefix stays resident while any referrer waits on the host."""
     L, H, D, e = (int(x) for x in golden["bpt_factors"])
     p = kvr.Pool(L, H, D, e, 8, 4096, 8 << 30, flags=kvr.METADATA_ONLY)
-    assert p.admit(0, 5400)[0] == kvr.OK
+    ctx, shared = int(golden["context_tokens"][0]), int(golden["shared_prefix_tokens"][0])
+    assert p.admit(0, shared)[0] == kvr.OK
     for rid in (1, 2, 3):
-        assert p.admit_sharing(rid, 8400, 0, 675)[0] == kvr.OK
+        assert p.admit_sharing(rid, ctx, 0, shared // 8)[0] == kvr.OK
     assert p.release(0) == kvr.OK                                           # the prefix outlives the request that made it
     assert p.suspend_to_host([1, 2, 3])[0] == kvr.OK
     s = p.stats()

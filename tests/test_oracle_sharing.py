@@ -59,7 +59,8 @@ def test_paper_sizes_metadata_only(golden):
     L, H, D, e = (int(x) for x in golden["bpt_factors"])
     BS, NB = 8, 4096
     p = orc.OrcPool(L, H, D, e, BS, NB, 8 << 30, with_data=False)
-    ctx, shared = int(golden["context_tokens"][0]), 5400
+    ctx, shared = int(golden["context_tokens"][0]), int(golden["shared_prefix_tokens"][0])
+    assert ctx - shared == int(golden["suffix_tokens"][0])
     assert p.admit(0, shared)[0] == orc.OK                                   # the system prefix, computed once
     st, blocks = p.admit_sharing(1, ctx, 0, shared // BS)
     assert st == orc.OK and blocks[:675].tolist() == p.info(0)[1]["blocks"].tolist()
