@@ -43,3 +43,34 @@ def test_plain_launch_with_gpus_2_starts_two_ranks_and_prints_one_line():
     assert d["n_gpus"] == 2 and d["dry_run"] is True and d["value"] is None and d["scaling"] == "weak"
     # 32 contexts of 8,400 tokens sharing 337 whole blocks (5,392 tokens): 3,008 private tokens each, on both ranks
     assert d["bookkeeping"]["bytes_suspended_per_step_all_ranks"] == 2 * 32 * 3008 * 80 * 2 * 128 * 2 * 2
+
+
+import pytest  # noqa: E402
+
+
+@pytest.mark.gpu
+def test_our_arm_prints_one_contract_line_on_a_gpu():
+    """`python bench.py` on a B200 (here the small configuration): one JSON line with the base keys, the roofline
+    and CPU-baseline objects, an end-to-end figure whose bytes really crossed the link, and kernels of our own."""
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--workload", "tiny", "--steps", "2", "--warmup", "3",
+                          "--no-extras"], capture_output=True, text=True, timeout=900)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [x for x in out.stdout.splitlines() if x.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                "vs_baseline", "dtype", "data", "config", "e2e", "gpu_launches", "clocks", "roofline", "cpu_baseline"):
+        assert key in d, key
+    assert d["n_gpus"] == 1 and d["steps"] == 2 and d["warmup"] == 3 and d["unit"] == "GB/s" and d["dtype"] == "u8"
+    assert d["config"]["workload"] == "tiny" and d["config"]["staging"]["library_default"] is True
+    r = d["roofline"]
+    assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["peak"] > 1000 and 0.2 < r["frac"] == pytest.approx(r["achieved"] / r["peak"])
+    assert r["traffic"] is not None and 0 < r["traffic"] <= r["algorithmic_bytes_per_launch"]
+    payload = d["config"]["payload_bytes_per_direction"]
+    assert d["e2e"]["d2h_bytes_per_step"] >= payload and d["e2e"]["h2d_bytes_per_step"] >= payload     # the bytes crossed the link
+    assert 0 < d["e2e"]["value"] <= d["value"] * 1.05 and d["gpu_launches"] >= 4
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] == 1 and d["cpu_baseline"]["value"] > 0
+    assert d["host_link"]["suspend_frac_of_d2h_peak"] > 0.5 and d["host_link"]["resume_frac_of_h2d_peak"] > 0.5

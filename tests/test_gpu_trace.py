@@ -26,15 +26,39 @@ def thresholds(lengths, bpt, host_cap):
     return lam, host_ttl(lam, c2, w_ref)
 
 
+class _RandomSync:
+    """The library pool with a seeded mix of call styles: moves are synchronous or left in flight, resumes ask for
+    low latency or not, and now and then the caller waits for everything.  Results must not depend on any of it."""
+
+    def __init__(self, pool, seed):
+        self._pool, self._rng = pool, np.random.default_rng(seed)
+
+    def suspend_to_host(self, ids):
+        return self._pool.suspend_to_host(ids, kvr.SYNC if self._rng.random() < 0.4 else 0)
+
+    def resume_from_host(self, ids):
+        flags = (kvr.SYNC if self._rng.random() < 0.4 else 0) | (kvr.LOW_LATENCY if self._rng.random() < 0.5 else 0)
+        return self._pool.resume_from_host(ids, flags)
+
+    def admit(self, rid, n):
+        if self._rng.random() < 0.1:
+            assert self._pool.wait() == kvr.OK
+        return self._pool.admit(rid, n)
+
+    def __getattr__(self, name):
+        return getattr(self._pool, name)
+
+
+@pytest.mark.parametrize("style", ["in-flight", "random-sync"])
 @pytest.mark.parametrize("mode", [dict(route=kvr.ROUTE_STAGED, kernel=kvr.KERNEL_BULK),
                                   dict(route=kvr.ROUTE_MAPPED, kernel=kvr.KERNEL_WARP)], ids=["staged-bulk", "mapped-warp"])
-def test_trace_small_geometry_with_data(mode):
+def test_trace_small_geometry_with_data(mode, style):
     geom = (2, 2, 16, 2, 4)                        # 64-byte rows, 256 bytes per token
     n_req, NB, host_cap = 160, 130, 160 * 4096
     lengths = context_lengths(("lognormal", 64, 0.6, 4, 400), n_req, 21)
     lam, ttl = thresholds(lengths, 256, host_cap)
     events, _ = event_trace(n_req, 21, lam, 60.0, ttl)
-    t = Twin(geom, NB, host_cap, seed=21, chunk_bytes=8192, staging_slots=2, **mode)
+    t = Twin(geom, NB, host_cap, seed=21, chunk_bytes=8192, staging_slots=2 if style == "in-flight" else 5, **mode)
     rng = np.random.default_rng(21)
     L, H, D, e, BS = geom
     o_view = t.o.data.reshape(2 * L, NB, BS * H * D * e)
@@ -51,7 +75,8 @@ def test_trace_small_geometry_with_data(mode):
     def after(name, args):
         if name == "suspend_to_host":
             t.assert_same_images(args[0])
-    counts = TraceRunner([t.o, t.g], lengths, fill=fill, after_call=after).run(events)
+    lib_pool = t.g if style == "in-flight" else _RandomSync(t.g, 5)
+    counts = TraceRunner([t.o, lib_pool], lengths, fill=fill, after_call=after).run(events)
     for k in ("offloaded", "resumed_resident", "resumed_from_host", "recomputed", "ttl_expired", "demoted"):
         assert counts.get(k, 0) > 0, (k, counts)
     t.assert_same_pool()
