@@ -475,6 +475,21 @@ kvr_status kvr_test_fail_nth(kvr_pool *pool, int32_t kind, int64_t n);
 int64_t kvr_test_points(kvr_pool *pool, int32_t kind);
 
 /*
+ * The staged route's planner on its own, for tests (no counterpart in the paper; pure host code).  Plans one move of
+ * n_items requests of n_tokens[i] tokens through a ring of `slots` slots of slot_bytes, of which one launch may
+ * cover launch_slots, starting at slot ring_next; resume != 0 plans a resume (flags: KVR_LOW_LATENCY); the
+ * single-launch thresholds may be 0 for the defaults.  Images are laid out one after another from offset 0 in
+ * 4096-byte granules.  Outputs (cap records each): chunks -- 6 numbers per launch: first slot, slots, payload bytes,
+ * copies, first segment, segments; copies -- 5 per link copy: launch, offset in the arena, offset in the ring,
+ * position inside the launch (unused bytes at the ring's end included), bytes; segs -- 5 per segment: byte offset of
+ * the request's block table among the tables, where image byte 0 would lie relative to the ring's base, first tile,
+ * tiles, blocks of the request; counts -- launches, copies, segments, the ring's next slot afterwards.
+ */
+kvr_status kvr_test_plan(const kvr_geometry *g, const int64_t *n_tokens, int32_t n_items, uint64_t slot_bytes, int32_t slots,
+                         int32_t launch_slots, int32_t ring_next, int32_t resume, uint32_t flags, uint64_t suspend_single_bytes,
+                         uint64_t resume_single_bytes, int64_t *chunks, int64_t *copies, int64_t *segs, int64_t cap, int64_t *counts);
+
+/*
  * Placement of the library's own arena (no counterpart in the paper).  Host DRAM is shared between the GPUs of a
  * node; each pool's arena is faulted in by threads bound to the CPUs of the NUMA node its GPU hangs off, so the
  * pages land next to that GPU's link.  kvr_pool_numa_node: the node used (-1: unknown, single-node host, caller's

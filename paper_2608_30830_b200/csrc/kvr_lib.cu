@@ -1748,6 +1748,64 @@ int64_t kvr_test_points(kvr_pool *p, int32_t kind) {
   return p->points[kind];
 }
 
+kvr_status kvr_test_plan(const kvr_geometry *g, const int64_t *n_tokens, int32_t n_items, uint64_t slot_bytes, int32_t slots,
+                         int32_t launch_slots, int32_t ring_next, int32_t resume, uint32_t flags, uint64_t suspend_single,
+                         uint64_t resume_single, int64_t *chunks, int64_t *copies, int64_t *segs, int64_t cap, int64_t *counts) {
+  const uint64_t bpt = kvr_bytes_per_token(g);
+  if (!bpt || !n_tokens || n_items < 0 || slots < 2 || launch_slots < 1 || launch_slots >= slots || ring_next < 0 ||
+      ring_next >= slots || !chunks || !copies || !segs || !counts || cap < 0)
+    return fail(KVR_ERR_INVALID_ARG, "kvr_test_plan: bad arguments");
+  try {
+    kvr_pool pool;                                  // bookkeeping fields only: the planner touches nothing else
+    kvr_pool *p = &pool;
+    p->bpt = bpt; p->row = (int)(bpt / 2 / g->layers); p->tile_bytes = p->row * g->block_size;
+    p->BS = g->block_size; p->planes = 2 * g->layers;
+    if (slot_bytes % 4096 || slot_bytes < (uint64_t)p->tile_bytes) return fail(KVR_ERR_INVALID_ARG, "kvr_test_plan: slot size");
+    p->slot_bytes = slot_bytes; p->launch_slots = launch_slots; p->call_flags = flags;
+    if (suspend_single) p->suspend_single = suspend_single;
+    if (resume_single) p->resume_single = resume_single;
+    Ring ring;
+    ring.base = reinterpret_cast<char *>(uintptr_t(1) << 40);   // never dereferenced
+    ring.slots.resize((size_t)slots);
+    ring.next = ring_next;
+    std::vector<Item> items;
+    uint64_t lin = 0, bt = 0;
+    for (int32_t i = 0; i < n_items; ++i) {
+      if (n_tokens[i] < 0) return fail(KVR_ERR_INVALID_ARG, "kvr_test_plan: negative length");
+      const int32_t nb = (int32_t)((n_tokens[i] + p->BS - 1) / p->BS);
+      items.push_back({(uint64_t)i, nullptr, nullptr, nb, n_tokens[i], lin, (size_t)bt, i, 0});
+      lin += align_up((uint64_t)n_tokens[i] * bpt, kArenaGranule);
+      bt += align_up((uint64_t)nb * 4, 16);
+    }
+    Plan pl;
+    plan_staged(p, items, ring, resume != 0, nullptr, pl);
+    int64_t n_copies = 0;
+    for (auto &ch : pl.chunks) n_copies += (int64_t)ch.copies.size();
+    counts[0] = (int64_t)pl.chunks.size(); counts[1] = n_copies; counts[2] = (int64_t)pl.segs.size(); counts[3] = pl.next_slot;
+    if ((int64_t)pl.chunks.size() > cap || n_copies > cap || (int64_t)pl.segs.size() > cap) return fail(KVR_ERR_INVALID_ARG, "kvr_test_plan: output arrays too small");
+    int64_t c = 0;
+    for (size_t k = 0; k < pl.chunks.size(); ++k) {
+      const Chunk &ch = pl.chunks[k];
+      int64_t *o = chunks + 6 * k;
+      o[0] = ch.first_slot; o[1] = ch.n_slots; o[2] = (int64_t)ch.bytes; o[3] = (int64_t)ch.copies.size(); o[4] = (int64_t)ch.seg_begin; o[5] = ch.nsegs;
+      for (auto &cp : ch.copies) {
+        int64_t *q = copies + 5 * c++;
+        q[0] = (int64_t)k; q[1] = (int64_t)cp.lin_off; q[2] = (int64_t)cp.ring_off; q[3] = (int64_t)cp.vpos; q[4] = (int64_t)cp.bytes;
+      }
+    }
+    for (size_t i = 0; i < pl.segs.size(); ++i) {
+      const Seg &sg = pl.segs[i];
+      int64_t *o = segs + 5 * i;
+      o[0] = (int64_t)reinterpret_cast<uintptr_t>(sg.bt);          // the item's table offset identifies the item
+      o[1] = (int64_t)(sg.img - ring.base);                        // where image byte 0 would lie, relative to the ring
+      o[2] = sg.tile_begin; o[3] = sg.tile_count; o[4] = sg.nb;
+    }
+    return KVR_OK;
+  } catch (const std::bad_alloc &) {
+    return fail(KVR_ERR_NOMEM, "out of host memory");
+  }
+}
+
 int32_t kvr_pool_numa_node(kvr_pool *p) { return p ? p->numa_node : -1; }
 
 kvr_status kvr_selftest_bounded_wait(kvr_pool *p, int32_t leave_error_set) {

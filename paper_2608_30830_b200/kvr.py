@@ -76,7 +76,7 @@ class Stats(C.Structure):
 
 EXPORTS = [
     "kvr_bytes_per_token", "kvr_pool_create", "kvr_pool_destroy", "kvr_request_admit", "kvr_request_admit_into", "kvr_request_release",
-    "kvr_request_admit_sharing", "kvr_request_admit_sharing_into", "kvr_request_sharing", "kvr_block_refcount", "kvr_test_fail_nth", "kvr_test_points",
+    "kvr_request_admit_sharing", "kvr_request_admit_sharing_into", "kvr_request_sharing", "kvr_block_refcount", "kvr_test_fail_nth", "kvr_test_points", "kvr_test_plan",
     "kvr_pool_numa_node", "kvr_numa_lookup",
     "kvr_retain_in_hbm", "kvr_suspend_to_host", "kvr_expire", "kvr_resume_from_host",
     "kvr_resume_from_host_into", "kvr_export_to_device", "kvr_import_from_device", "kvr_request_info",
@@ -128,6 +128,9 @@ def lib():
     L.kvr_test_fail_nth.argtypes = [vp, i32, i64]
     L.kvr_test_points.restype = i64
     L.kvr_test_points.argtypes = [vp, i32]
+    L.kvr_test_plan.restype = i32
+    L.kvr_test_plan.argtypes = [C.POINTER(Geometry), C.POINTER(i64), i32, u64, i32, i32, i32, i32, u32, u64, u64,
+                                C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), i64, C.POINTER(i64)]
     L.kvr_pool_numa_node.restype = i32
     L.kvr_pool_numa_node.argtypes = [vp]
     L.kvr_numa_lookup.restype = i32
@@ -295,6 +298,25 @@ class Controller:
 def read_load(device_buf, nbytes, launches, device_sink, stream=None):
     """kvr_read_load: enqueue the synthetic HBM-read load (benchmark support)."""
     return lib().kvr_read_load(device_buf, nbytes, launches, device_sink, stream)
+
+
+def test_plan(geom, n_tokens, slot_bytes, slots, launch_slots, ring_next=0, resume=False, flags=0, suspend_single=0,
+              resume_single=0, cap=1 << 16):
+    """kvr_test_plan: the staged route's plan for one move, as numpy arrays (chunks[k, 6], copies[j, 5], segs[i, 5])
+    and the ring's next slot."""
+    g = Geometry(*geom)
+    n = np.ascontiguousarray(n_tokens, dtype=np.int64)
+    chunks, copies, segs = (np.zeros((cap, w), dtype=np.int64) for w in (6, 5, 5))
+    counts = np.zeros(4, dtype=np.int64)
+    p64 = lambda a: a.ctypes.data_as(C.POINTER(C.c_int64))   # noqa: E731
+    st = lib().kvr_test_plan(C.byref(g), p64(n), len(n), slot_bytes, slots, launch_slots, ring_next, int(resume), flags,
+                             suspend_single, resume_single, p64(chunks), p64(copies), p64(segs), cap, p64(counts))
+    if st != OK:
+        raise KvrError(st, last_error())
+    return chunks[:counts[0]].copy(), copies[:counts[1]].copy(), segs[:counts[2]].copy(), int(counts[3])
+
+
+test_plan.__test__ = False      # a library call, not a pytest test
 
 
 def numa_lookup(sysfs_root, pci_bus_id, cap=4096):
