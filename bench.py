@@ -556,7 +556,13 @@ def run_ours(args):
         for i in range(0, view.numel(), step_elems):
             view[i:i + step_elems].normal_(generator=gen)
         torch.cuda.synchronize()
-        dev_arena = torch.empty(host_cap, dtype=torch.uint8, device="cuda") if args.arena == "device" else None
+        dev_arena = None
+        if args.arena == "device":
+            dev_arena = torch.empty(host_cap, dtype=torch.uint8, device="cuda")
+        elif args.arena == "peer":               # the next GPU's memory, reached over NVLink (needs a second GPU)
+            if torch.cuda.device_count() < 2 or world > 1:
+                raise SystemExit("--arena peer needs a second GPU and a single-rank run")
+            dev_arena = torch.empty(host_cap, dtype=torch.uint8, device="cuda:%d" % ((local + 1) % torch.cuda.device_count()))
         pool = kvr.Pool(*w.geom, w.num_blocks, host_cap, initial_free_order=free_order(seed, w.num_blocks),
                         device=local, device_pool=dev_pool.data_ptr(), route=route,
                         host_arena=dev_arena.data_ptr() if dev_arena is not None else None,
@@ -768,6 +774,9 @@ def run_ours(args):
         if link is None:        # device-memory tier: no host link on the path; the bound is HBM
             host_link = {"arena": "device memory", "suspend_gbs": sus_gbs, "resume_gbs": res_gbs,
                          "suspend_frac_of_hbm_peak": 2 * sus_gbs / world / peak, "resume_frac_of_hbm_peak": 2 * res_gbs / world / peak}
+            if args.arena == "peer":             # bound by NVLink: 770 GB/s per direction measured for a peer copy on this machine
+                host_link = {"arena": "peer GPU memory over NVLink", "suspend_gbs": sus_gbs, "resume_gbs": res_gbs,
+                             "suspend_frac_of_peer_copy_770": sus_gbs / 770.0, "resume_frac_of_peer_copy_770": res_gbs / 770.0}
         else:
             host_link = dict(link)
             d2h_sum = sum(r["d2h_alone_gbs"] for r in per_rank_links)
@@ -846,8 +855,8 @@ def main():
     ap.add_argument("--copy-piece-mib", type=int, default=int(os.environ.get("KVR_COPY_PIECE_MIB", "0")),
                     help="largest single link copy (0 = library default, 64)")
     ap.add_argument("--bulk-shape", default=os.environ.get("KVR_BULK_SHAPE", ""), help="bulk mover shape: warps,stages,piece_bytes")
-    ap.add_argument("--arena", default="host", choices=["host", "device"],
-                    help="where the second tier lives: pinned host memory, or device memory (stand-in for a peer GPU)")
+    ap.add_argument("--arena", default="host", choices=["host", "device", "peer"],
+                    help="where the second tier lives: pinned host memory, this GPU's memory (stand-in for a peer), or the next GPU's")
     ap.add_argument("--max-ctas", type=int, default=0, help="cap on the movers' grid (0 = fill the GPU)")
     ap.add_argument("--num-blocks", type=int, default=0, help="shrink the pool (profiling captures)")
     ap.add_argument("--requests", type=int, default=0, help="override the request count")

@@ -296,6 +296,37 @@ def test_arena_in_device_memory(route):
     t.close()
 
 
+@pytest.mark.parametrize("route", [kvr.ROUTE_STAGED, kvr.ROUTE_MAPPED])
+def test_arena_in_a_peer_gpus_memory(route):
+    """The same with the arena on another GPU (the peer-HBM tier over NVLink): the library enables peer access, the
+    copies follow the pointer and the direct route's kernels use plain loads, stores and non-multicast bulk copies.
+    Needs two GPUs: skipped on a one-GPU machine."""
+    if torch.cuda.device_count() < 2:
+        pytest.skip("needs two GPUs")
+    if not torch.cuda.can_device_access_peer(0, 1):
+        pytest.skip("GPU 0 cannot address GPU 1")
+    geom = (4, 2, 64, 2, 16)
+    cap = 1 << 21
+    arena = torch.zeros(cap, dtype=torch.uint8, device="cuda:1")
+    torch.cuda.synchronize(1)
+    t = Twin(geom, 96, cap, seed=15, host_arena=arena.data_ptr(), route=route, chunk_bytes=65536, staging_slots=3)
+    lens = [500, 123, 16, 0, 77]
+    ids = list(range(len(lens)))
+    for rid, n in zip(ids, lens):
+        assert t.both("admit", rid, n)[1][0] == kvr.OK
+    a, b = t.both("suspend_to_host", ids)
+    assert a == b and t.g.wait() == kvr.OK
+    peer = arena.cpu().numpy()
+    for rid in ids:
+        d = t.o.info(rid)[1]
+        off = t.g.info(rid)[1]["arena_offset"]
+        assert off == d["arena_offset"] and np.array_equal(peer[off:off + d["image_bytes"]], d["image"])
+    a, b = t.both("resume_from_host", ids[::-1])
+    assert a == b
+    t.assert_same_pool()
+    t.close()
+
+
 @pytest.mark.parametrize("mode", MODES)
 def test_guard_bands_stay_intact(mode):
     """Canary regions directly before and after the caller-owned pool and arena must survive a busy script:
