@@ -6,8 +6,8 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 SO = os.path.join(PKG, "libkvr.so")
-SOURCES = ["kvr_kernels.cu", "kvr_lib.cu", "kvr_noalloc.cu", "kvr_policy.cpp", "kvr_controller.cpp", "kvr_numa.cpp"]
-DEPS = SOURCES + ["kvr_kernels.cuh", "kvr_meta.hpp", "kvr_numa.hpp", os.path.join("..", "..", "include", "kvr.h")]
+SOURCES = ["kvr_kernels.cu", "kvr_engine.cu", "kvr_lib.cu", "kvr_noalloc.cu", "kvr_policy.cpp", "kvr_controller.cpp", "kvr_numa.cpp"]
+DEPS = SOURCES + ["kvr_kernels.cuh", "kvr_meta.hpp", "kvr_numa.hpp", "kvr_pool.hpp", os.path.join("..", "..", "include", "kvr.h")]
 
 
 def stale():
