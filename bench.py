@@ -462,10 +462,14 @@ def run_trace(args):
                   "outcomes": {"%s:%d" % k: v for k, v in sorted(outcomes.items())},
                   "gpu_cost_per_request": cs["gpu_cost"] / w.n_requests},
         "roofline": {"bound": "hbm", "peak": peak, "unit": "GB/s", "gather_frac": g_gbs / peak, "scatter_frac": s_gbs / peak,
+                     "gather_in_kernel_frac": 2 * st["gather_bytes"] / max(st["gather_kernel_ms"], 1e-9) / 1e6 / peak,
+                     "scatter_in_kernel_frac": 2 * st["scatter_bytes"] / max(st["scatter_kernel_ms"], 1e-9) / 1e6 / peak,
                      "gather_launches": int(st["gather_launches"]), "scatter_launches": int(st["scatter_launches"]),
                      "mover_busy_us_per_gb": {"gather": 1e3 * st["gather_ms"] / max(st["gather_bytes"] / 1e9, 1e-9),
                                               "scatter": 1e3 * st["scatter_ms"] / max(st["scatter_bytes"] / 1e9, 1e-9)},
-                     "note": "per-request moves of ~0.6 GiB: launches are smaller than in the batched configurations"},
+                     "note": "per-request moves of ~0.6 GiB, one launch each; *_frac is taken from CUDA events around every launch "
+                             "(they include the tens of microseconds a completion takes while the copy engine is busy), "
+                             "*_in_kernel_frac from the kernels' own first and last clock stamps"},
         "host_link": link, "clocks": clocks, "gpu_launches": int(st["gather_launches"] + st["scatter_launches"]),
     }
     print(json.dumps(out))
