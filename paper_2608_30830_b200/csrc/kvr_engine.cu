@@ -90,10 +90,10 @@ static void retire(kvr_pool *p, Op &op) {
   }
   if (op.desc >= 0 && op.n_stamps) {
     // first CTA start to last CTA end of every launch, as the kernels stamped them
-    const unsigned long long *st = reinterpret_cast<const unsigned long long *>(p->descs[op.desc].h + op.stamp_off);
+    const LaunchRec *rec = reinterpret_cast<const LaunchRec *>(p->descs[op.desc].h + op.stamp_off);
     double ms = 0;
     for (int i = 0; i < op.n_stamps; ++i)
-      if (st[2 * i + 1] > st[2 * i]) ms += (double)(st[2 * i + 1] - st[2 * i]) * 1e-6;
+      if (rec[i].last_end > rec[i].first_start) ms += (double)(rec[i].last_end - rec[i].first_start) * 1e-6;
     if (op.kind == OP_SUSPEND || op.kind == OP_EXPORT) p->st.gather_kernel_ms += ms; else p->st.scatter_kernel_ms += ms;
   }
   for (auto e : op.chunk_done) put_event(p, e);
@@ -306,11 +306,13 @@ static void plan_direct(kvr_pool *p, const std::vector<Item> &items, char *lin_b
 }
 
 static kvr_status launch(kvr_pool *p, bool gather, const Seg *segs_dev, const Chunk &c, cudaStream_t s, Op &op,
-                  unsigned long long *stamp) {
+                  LaunchRec *rec_dev) {
   MoveArgs a{};
   a.segs = segs_dev + c.seg_begin; a.nsegs = c.nsegs; a.total_tiles = c.tiles;
   a.pool = p->d_pool; a.plane_stride = p->plane_stride; a.block_stride = p->block_stride; a.tile_bytes = p->tile_bytes;
-  a.row_bytes = p->row; a.block_size = p->BS; a.num_blocks = p->NB; a.status = p->status_word; a.stamp = stamp;
+  a.row_bytes = p->row; a.block_size = p->BS; a.num_blocks = p->NB; a.status = p->status_word;
+  a.stamp = p->profile ? &rec_dev->first_start : nullptr;
+  a.work = &rec_dev->work;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   if (p->profile) {
     kvr_status s0 = get_event(p, &e0); if (s0) return s0;
@@ -402,7 +404,7 @@ static kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> 
   if (route == KVR_ROUTE_DMA2D) return enqueue_dma2d(p, op, items, to_linear, block_tag, arena_waits, t_call, out_seq);
 
   // plan with table addresses relative to the descriptor buffer, then size the buffer exactly:
-  // [block tables][segments][stamps]
+  // [block tables][segments][one record per launch: work counter and time stamps]
   size_t bt_bytes = 0;
   for (auto &it : items) { it.bt_off = bt_bytes; bt_bytes += align_up((uint64_t)it.nb * 4, 16); }
   Plan pl;
@@ -414,9 +416,9 @@ static kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> 
     plan_direct(p, items, route == KVR_ROUTE_MAPPED ? p->arena_dev : lin_dev, nullptr, pl);
   }
   const size_t seg_off = align_up(bt_bytes, 64);
-  const size_t stamp_off = align_up(seg_off + pl.segs.size() * sizeof(Seg), 64);
-  const int n_stamps = p->profile ? (int)pl.chunks.size() : 0;
-  size_t desc_bytes = n_stamps ? stamp_off + 16 * (size_t)n_stamps : seg_off + pl.segs.size() * sizeof(Seg);
+  const size_t rec_off = align_up(seg_off + pl.segs.size() * sizeof(Seg), 64);
+  const int n_recs = (int)pl.chunks.size();
+  size_t desc_bytes = rec_off + sizeof(LaunchRec) * (size_t)n_recs;
   if (!desc_bytes) desc_bytes = 64;
   if (lease >= 0 && p->descs[lease].cap >= desc_bytes) {
     op.desc = lease;
@@ -434,12 +436,9 @@ static kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> 
   }
   DescBuf &db = p->descs[op.desc];
   db.busy = op.seq;
-  for (int i = 0; i < n_stamps; ++i) {
-    unsigned long long *st = reinterpret_cast<unsigned long long *>(db.h + stamp_off) + 2 * i;
-    st[0] = ~0ull; st[1] = 0;
-  }
-  op.stamp_off = stamp_off; op.n_stamps = n_stamps;
-  unsigned long long *stamps_dev = n_stamps ? reinterpret_cast<unsigned long long *>(db.d + stamp_off) : nullptr;
+  for (int i = 0; i < n_recs; ++i) reinterpret_cast<LaunchRec *>(db.h + rec_off)[i] = LaunchRec{~0ull, 0, 0, 0};
+  op.stamp_off = rec_off; op.n_stamps = p->profile ? n_recs : 0;
+  LaunchRec *recs_dev = reinterpret_cast<LaunchRec *>(db.d + rec_off);
   for (auto &it : items) if (it.nb) memcpy(db.h + it.bt_off, it.blocks, (size_t)it.nb * 4);
   for (auto &sg : pl.segs) sg.bt = reinterpret_cast<const int32_t *>(db.d + reinterpret_cast<uintptr_t>(sg.bt));
   if (!pl.segs.empty()) memcpy(db.h + seg_off, pl.segs.data(), pl.segs.size() * sizeof(Seg));
@@ -506,7 +505,7 @@ static kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> 
     alloc_point(p);
     op.chunk_done.push_back(cd);
     if (!staged) {
-      if ((s = launch(p, to_linear, segs_dev, ch, k, op, stamps_dev ? stamps_dev + 2 * ci : nullptr))) return s;
+      if ((s = launch(p, to_linear, segs_dev, ch, k, op, recs_dev + ci))) return s;
       CUP(p, cudaEventRecord(cd, k));
       continue;
     }
@@ -533,7 +532,7 @@ static kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> 
         if (sl.used && (!latest || sl.seq > latest->seq)) latest = &sl;
       }
       if (latest) CUP(p, cudaStreamWaitEvent(k, ring->slots[latest->owner].freed, 0));
-      if ((s = launch(p, true, segs_dev, ch, k, op, stamps_dev ? stamps_dev + 2 * ci : nullptr))) return s;
+      if ((s = launch(p, true, segs_dev, ch, k, op, recs_dev + ci))) return s;
       CUP(p, cudaEventRecord(filled, k));
       CUP(p, cudaStreamWaitEvent(c, filled, 0));
       // the copies go out in pieces: one very large cudaMemcpyAsync to pinned memory sustains less than the same
@@ -580,7 +579,7 @@ static kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> 
         }
       CUP(p, cudaEventRecord(filled, c));
       CUP(p, cudaStreamWaitEvent(k, filled, 0));
-      if ((s = launch(p, false, segs_dev, ch, k, op, stamps_dev ? stamps_dev + 2 * ci : nullptr))) return s;
+      if ((s = launch(p, false, segs_dev, ch, k, op, recs_dev + ci))) return s;
       if ((s = release(0, ch.n_slots, k))) return s;       // the scatter has read every slot of the chunk
       CUP(p, cudaEventRecord(cd, k));
     }
@@ -591,8 +590,8 @@ static kvr_status enqueue_impl(kvr_pool *p, Op &op, int kind, std::vector<Item> 
   cudaStream_t reader = staged ? (to_linear ? k : c) : k;
   CUP(p, cudaEventRecord(op.read_done, reader));
   if (first != last) CUP(p, cudaStreamWaitEvent(last, op.read_done, 0));   // `done` must also cover the first stream (e.g. an empty move)
-  if (n_stamps)      // the stamps come back with the move: `last` is ordered after every launch
-    CUP(p, cudaMemcpyAsync(db.h + stamp_off, db.d + stamp_off, 16 * (size_t)n_stamps, cudaMemcpyDeviceToHost, last));
+  if (op.n_stamps)   // the stamps come back with the move: `last` is ordered after every launch
+    CUP(p, cudaMemcpyAsync(db.h + rec_off, db.d + rec_off, sizeof(LaunchRec) * (size_t)n_recs, cudaMemcpyDeviceToHost, last));
   CUP(p, cudaEventRecord(op.done, last));
 
   if (staged) ring->next = pl.next_slot;

@@ -12,6 +12,14 @@
 //   move_bulk : one thread per pipeline drives bulk async copies
 //               global -> shared -> global through a ring of shared-memory
 //               stages guarded by mbarriers (no multicast: no tile is shared)
+//
+// Work is handed out dynamically: a launch carries a zeroed counter and every
+// pipeline (or warp) takes the next unit with one atomicAdd when it is free.
+// SMs do not all reach HBM equally fast, so fixed equal shares leave most of
+// the chip idle while the slowest SM finishes (measured: 6.2 TB/s with equal
+// shares, 6.7-6.8 TB/s with the counter, on 2-4 GiB launches); claiming one
+// unit at a time also keeps all pipelines inside one moving window of the
+// image.
 #include "kvr_kernels.cuh"
 
 namespace kvr {
@@ -89,9 +97,9 @@ __device__ __forceinline__ Tile locate(const MoveArgs &a, const long long *cum, 
 
 // ---- warp mover --------------------------------------------------------------------
 
-// One warp per tile; consecutive warps take consecutive tiles, so at any moment the grid covers one
-// contiguous window of the image.  A lane keeps 8 independent 16-byte loads in flight (streaming cache
-// policy: every byte is touched once) before it stores them.
+// One warp per tile; the warps of the grid take consecutive tiles (by the launch's work counter when there is one,
+// else grid-strided), so at any moment the grid covers one contiguous window of the image.  A lane keeps 8
+// independent 16-byte loads in flight (streaming cache policy: every byte is touched once) before it stores them.
 template <bool GATHER>
 __global__ void __launch_bounds__(kWarpThreads) move_warp_kernel(const MoveArgs a) {
   // (nsegs + 1) prefix sums, sized at launch (typically a few dozen bytes)
@@ -101,7 +109,17 @@ __global__ void __launch_bounds__(kWarpThreads) move_warp_kernel(const MoveArgs 
   const int lane = threadIdx.x & 31;
   const int warps_per_cta = blockDim.x >> 5;
   const long long stride = (long long)gridDim.x * warps_per_cta;
-  for (long long w = (long long)blockIdx.x * warps_per_cta + (threadIdx.x >> 5); w < a.total_tiles; w += stride) {
+  long long next = (long long)blockIdx.x * warps_per_cta + (threadIdx.x >> 5);
+  for (;;) {
+    long long w;
+    if (a.work) {
+      unsigned long long claimed = 0;
+      if (lane == 0) claimed = atomicAdd(a.work, 1ull);
+      w = (long long)__shfl_sync(0xffffffffu, claimed, 0);
+    } else {
+      w = next; next += stride;
+    }
+    if (w >= a.total_tiles) break;
     const Tile t = locate(a, cum, w);
     const uint4 *src = reinterpret_cast<const uint4 *>(GATHER ? t.pool_ptr : t.lin_ptr);
     uint4 *dst = reinterpret_cast<uint4 *>(GATHER ? t.lin_ptr : t.pool_ptr);
@@ -161,7 +179,8 @@ __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.w
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // STAGES shared-memory stages per pipeline; a store trails its load by LAG = STAGES/2 units,
-// so LAG loads and STAGES-LAG stores are in flight per pipeline.
+// so LAG loads and STAGES-LAG stores are in flight per pipeline.  A pipeline takes its units from the launch's
+// work counter, one at a time.
 template <bool GATHER, int STAGES>
 __global__ void __launch_bounds__(kMaxBulkWarps * 32) move_bulk_kernel(const MoveArgs a, const int piece_bytes) {
   constexpr int LAG = STAGES / 2 > 0 ? STAGES / 2 : 1;
@@ -185,40 +204,48 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32) move_bulk_kernel(const Mov
   const int warps_per_cta = blockDim.x >> 5;
   const int pieces_per_tile = (a.tile_bytes + piece_bytes - 1) / piece_bytes;
   const long long total_units = a.total_tiles * pieces_per_tile;
-  // every pipeline takes one contiguous, equally long run of units
+  // without a work counter every pipeline takes one contiguous, equally long run of units
   const long long pipe = (long long)blockIdx.x * warps_per_cta + warp;
   const long long n_pipes = (long long)gridDim.x * warps_per_cta;
   const long long per = total_units / n_pipes, extra = total_units - per * n_pipes;
-  const long long u0 = pipe * per + (pipe < extra ? pipe : extra);
-  const long long n = per + (pipe < extra ? 1 : 0);
+  long long fixed_next = pipe * per + (pipe < extra ? pipe : extra);
+  const long long fixed_end = fixed_next + per + (pipe < extra ? 1 : 0);
   unsigned char *my_ring = ring + (size_t)warp * STAGES * piece_bytes;
   unsigned phase_bits = 0;
-  bool failed = false;
+  bool failed = false, more = true;
+  long long issued = 0, stored = 0;      // units whose load / store this pipeline has issued
 
-  for (long long it = 0; it < n + LAG && !failed; ++it) {
-    if (it < n) {
-      const int stage = (int)(it % STAGES);
-      // the store that last read this stage (unit it - STAGES) must be done with shared memory
-      if (it >= STAGES) bulk_wait_read<STAGES - LAG - 1>();
-      const long long u = u0 + it;
-      const long long w = u / pieces_per_tile;
-      const int off = (int)(u - w * pieces_per_tile) * piece_bytes;
-      const Tile t = locate(a, cum, w);
-      int len = t.bytes - off;
-      if (len > piece_bytes) len = piece_bytes;
-      if (len < 0) len = 0;
-      pend_len[warp][stage] = len;
-      pend_dst[warp][stage] = (GATHER ? t.lin_ptr : t.pool_ptr) + off;
-      if (len > 0) {
-        const unsigned bar = smem_addr(&bars[warp][stage]);
-        mbar_expect_tx(bar, (unsigned)len);
-        bulk_load(smem_addr(my_ring + (size_t)stage * piece_bytes), (GATHER ? t.pool_ptr : t.lin_ptr) + off,
-                  (unsigned)len, bar);
+  // Every turn issues the load of one more unit while there is one, and the store of the unit LAG behind it.
+  for (;;) {
+    if (more) {
+      long long u;
+      if (a.work) u = (long long)atomicAdd(a.work, 1ull);
+      else u = fixed_next < fixed_end ? fixed_next++ : total_units;
+      if (u >= total_units) {
+        more = false;
+      } else {
+        const int stage = (int)(issued % STAGES);
+        // the store that last read this stage (STAGES units back) must be done with shared memory
+        if (issued >= STAGES) bulk_wait_read<STAGES - LAG - 1>();
+        const long long w = u / pieces_per_tile;
+        const int off = (int)(u - w * pieces_per_tile) * piece_bytes;
+        const Tile t = locate(a, cum, w);
+        int len = t.bytes - off;
+        if (len > piece_bytes) len = piece_bytes;
+        if (len < 0) len = 0;
+        pend_len[warp][stage] = len;
+        pend_dst[warp][stage] = (GATHER ? t.lin_ptr : t.pool_ptr) + off;
+        if (len > 0) {
+          const unsigned bar = smem_addr(&bars[warp][stage]);
+          mbar_expect_tx(bar, (unsigned)len);
+          bulk_load(smem_addr(my_ring + (size_t)stage * piece_bytes), (GATHER ? t.pool_ptr : t.lin_ptr) + off,
+                    (unsigned)len, bar);
+        }
+        ++issued;
       }
     }
-    const long long j = it - LAG;
-    if (j >= 0 && j < n) {
-      const int stage = (int)(j % STAGES);
+    if (issued - stored > LAG || (!more && stored < issued)) {
+      const int stage = (int)(stored % STAGES);
       const int len = pend_len[warp][stage];
       if (len > 0) {
         if (!mbar_wait(smem_addr(&bars[warp][stage]), (phase_bits >> stage) & 1u)) { failed = true; break; }
@@ -226,7 +253,9 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32) move_bulk_kernel(const Mov
         bulk_store(pend_dst[warp][stage], smem_addr(my_ring + (size_t)stage * piece_bytes), (unsigned)len);
       }
       bulk_commit();   // one group per unit, empty or not, so the group arithmetic above holds
+      ++stored;
     }
+    if (!more && stored == issued) break;
   }
   if (failed) {
     *reinterpret_cast<volatile int *>(a.status) = 1;   // pinned host word, read by the host

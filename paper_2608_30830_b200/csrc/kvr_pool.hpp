@@ -68,7 +68,7 @@ struct Op {
   std::vector<ReqDone> reqs;                        // request -> index of the chunk that completes it (-1: none)
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof;   // kernel brackets (KVR_PROFILE)
   int desc = -1;
-  size_t stamp_off = 0; int n_stamps = 0;           // in-kernel time stamps inside the descriptor buffer (KVR_PROFILE)
+  size_t stamp_off = 0; int n_stamps = 0;           // launch records inside the descriptor buffer whose stamps are read back (KVR_PROFILE)
   double host_ms = 0;
 };
 
@@ -94,6 +94,10 @@ struct Item {
   int32_t batch_index;     // position in the caller's batch (per_req)
   int32_t prev_state;      // state to go back to if the move cannot be enqueued
 };
+
+// One per mover launch, inside the move's descriptor buffer: the kernel's work counter (uploaded as zero) and, under
+// KVR_PROFILE, the earliest start and latest end any of its CTAs stamped (%globaltimer nanoseconds).
+struct LaunchRec { unsigned long long first_start, last_end, work, pad; };
 
 struct CopyCmd { uint64_t lin_off; uint64_t ring_off; uint64_t vpos; uint64_t bytes; };
 struct Chunk {
