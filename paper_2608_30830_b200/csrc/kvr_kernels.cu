@@ -14,7 +14,8 @@
 //               stages guarded by mbarriers (no multicast: no tile is shared)
 //
 // Work is handed out dynamically: a launch carries a zeroed counter and every
-// pipeline (or warp) takes the next unit with one atomicAdd when it is free.
+// pipeline (or warp) takes the next unit (32 KiB, or a few smaller ones) with
+// one atomicAdd when it is free.
 // SMs do not all reach HBM equally fast, so fixed equal shares leave most of
 // the chip idle while the slowest SM finishes (measured: 6.2 TB/s with equal
 // shares, 6.7-6.8 TB/s with the counter, on 2-4 GiB launches); claiming one
@@ -30,6 +31,7 @@ constexpr int kWarpThreads = 256;          // threads per CTA of the warp mover
 constexpr int kMaxBulkWarps = 8;
 constexpr int kMaxBulkStages = 8;
 constexpr unsigned kSpinLimit = 1u << 22;  // bounded mbarrier wait (each spin sleeps >= 32 ns after the first 64)
+constexpr int kClaimBytes = 32 * 1024;     // work taken from a launch's counter per atomicAdd (at least one unit)
 
 // Exclusive prefix sum of tile counts into cum[0..nsegs]; cum[nsegs] = total.
 // Done by warp 0 in strides of 32 with shuffle-up, carrying the running total.
@@ -110,12 +112,19 @@ __global__ void __launch_bounds__(kWarpThreads) move_warp_kernel(const MoveArgs 
   const int warps_per_cta = blockDim.x >> 5;
   const long long stride = (long long)gridDim.x * warps_per_cta;
   long long next = (long long)blockIdx.x * warps_per_cta + (threadIdx.x >> 5);
+  // small tiles are claimed several at a time, so that the counter is not the bottleneck
+  const int claim = a.tile_bytes >= kClaimBytes ? 1 : kClaimBytes / a.tile_bytes;
+  long long claim_end = 0;
   for (;;) {
     long long w;
     if (a.work) {
-      unsigned long long claimed = 0;
-      if (lane == 0) claimed = atomicAdd(a.work, 1ull);
-      w = (long long)__shfl_sync(0xffffffffu, claimed, 0);
+      if (next >= claim_end) {
+        unsigned long long first = 0;
+        if (lane == 0) first = atomicAdd(a.work, (unsigned long long)claim);
+        next = (long long)__shfl_sync(0xffffffffu, first, 0);
+        claim_end = next + claim;
+      }
+      w = next++;
     } else {
       w = next; next += stride;
     }
@@ -214,13 +223,23 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32) move_bulk_kernel(const Mov
   unsigned phase_bits = 0;
   bool failed = false, more = true;
   long long issued = 0, stored = 0;      // units whose load / store this pipeline has issued
+  // small pieces are claimed several at a time, so that the counter is not the bottleneck
+  const int claim = piece_bytes >= kClaimBytes ? 1 : kClaimBytes / piece_bytes;
+  long long claim_next = 0, claim_end = 0;
 
   // Every turn issues the load of one more unit while there is one, and the store of the unit LAG behind it.
   for (;;) {
     if (more) {
       long long u;
-      if (a.work) u = (long long)atomicAdd(a.work, 1ull);
-      else u = fixed_next < fixed_end ? fixed_next++ : total_units;
+      if (a.work) {
+        if (claim_next >= claim_end) {
+          claim_next = (long long)atomicAdd(a.work, (unsigned long long)claim);
+          claim_end = claim_next + claim;
+        }
+        u = claim_next++;
+      } else {
+        u = fixed_next < fixed_end ? fixed_next++ : total_units;
+      }
       if (u >= total_units) {
         more = false;
       } else {
