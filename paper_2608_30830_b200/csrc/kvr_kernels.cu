@@ -210,15 +210,8 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32) move_bulk_kernel(const Mov
   scan_segments(a, cum);   // ends with __syncthreads()
   if (lane != 0) return;
 
-  const int warps_per_cta = blockDim.x >> 5;
   const int pieces_per_tile = (a.tile_bytes + piece_bytes - 1) / piece_bytes;
   const long long total_units = a.total_tiles * pieces_per_tile;
-  // without a work counter every pipeline takes one contiguous, equally long run of units
-  const long long pipe = (long long)blockIdx.x * warps_per_cta + warp;
-  const long long n_pipes = (long long)gridDim.x * warps_per_cta;
-  const long long per = total_units / n_pipes, extra = total_units - per * n_pipes;
-  long long fixed_next = pipe * per + (pipe < extra ? pipe : extra);
-  const long long fixed_end = fixed_next + per + (pipe < extra ? 1 : 0);
   unsigned char *my_ring = ring + (size_t)warp * STAGES * piece_bytes;
   unsigned phase_bits = 0;
   bool failed = false, more = true;
@@ -231,15 +224,11 @@ __global__ void __launch_bounds__(kMaxBulkWarps * 32) move_bulk_kernel(const Mov
   for (;;) {
     if (more) {
       long long u;
-      if (a.work) {
-        if (claim_next >= claim_end) {
-          claim_next = (long long)atomicAdd(a.work, (unsigned long long)claim);
-          claim_end = claim_next + claim;
-        }
-        u = claim_next++;
-      } else {
-        u = fixed_next < fixed_end ? fixed_next++ : total_units;
+      if (claim_next >= claim_end) {
+        claim_next = (long long)atomicAdd(a.work, (unsigned long long)claim);
+        claim_end = claim_next + claim;
       }
+      u = claim_next++;
       if (u >= total_units) {
         more = false;
       } else {
@@ -396,7 +385,7 @@ cudaError_t bulk_configure(const BulkShape &sh) {
 cudaError_t launch_move_bulk(bool gather, const MoveArgs &a, const BulkShape &sh, int grid_limit, int sm_count,
                              cudaStream_t s) {
   if (a.total_tiles <= 0) return cudaSuccess;
-  if (a.nsegs < 1 || a.nsegs > kMaxSegs) return cudaErrorInvalidValue;
+  if (a.nsegs < 1 || a.nsegs > kMaxSegs || !a.work) return cudaErrorInvalidValue;
   const size_t smem = (size_t)sh.warps * sh.stages * sh.piece_bytes;
   const int pieces_per_tile = (a.tile_bytes + sh.piece_bytes - 1) / sh.piece_bytes;
   const long long units = a.total_tiles * pieces_per_tile;

@@ -36,9 +36,9 @@ struct MoveArgs {
   int *status;           // DEVICE or NULL: error word (0 = fine); 1 = a bounded wait ran out, 3 = a table entry out of range
   unsigned long long *stamp;  // DEVICE or NULL: stamp[0] = earliest start, stamp[1] = latest end of any CTA, in
                               // %globaltimer nanoseconds (the host initialises them to ~0 and 0)
-  unsigned long long *work;   // DEVICE or NULL: work counter of this launch, zero when the kernel starts.  With it the
-                              // movers hand out work one unit at a time (whoever is free takes the next tile), so all
-                              // SMs finish together; without it every pipeline or warp takes a fixed share.
+  unsigned long long *work;   // DEVICE: work counter of this launch, zero when the kernel starts.  The movers hand out
+                              // work through it (whoever is free takes the next unit), so all SMs finish together.  The
+                              // bulk mover needs it; the warp mover falls back to a grid-strided loop when it is NULL.
 };
 
 struct BulkShape {       // tuning of the bulk mover

@@ -817,6 +817,7 @@ kvr_status kvr_selftest_block_check(kvr_pool *p, int32_t leave_error_set) {
   // to be one block shorter: the entry is out of range for the kernel, yet inside the real allocation, so even a
   // broken check could not make the launch touch memory that is not the pool's.
   reinterpret_cast<int32_t *>(db.h)[0] = p->NB - 1;
+  *reinterpret_cast<unsigned long long *>(db.h + 32) = 0;          // the launch's work counter
   Seg sg{};
   sg.bt = reinterpret_cast<const int32_t *>(db.d);
   sg.img = p->out_ring.base;
@@ -827,6 +828,7 @@ kvr_status kvr_selftest_block_check(kvr_pool *p, int32_t leave_error_set) {
   a.segs = reinterpret_cast<const Seg *>(db.d + 64); a.nsegs = 1; a.total_tiles = 1;
   a.pool = p->d_pool; a.plane_stride = p->plane_stride; a.block_stride = p->block_stride; a.tile_bytes = p->tile_bytes;
   a.row_bytes = p->row; a.block_size = p->BS; a.num_blocks = p->NB - 1; a.status = p->status_word;
+  a.work = reinterpret_cast<unsigned long long *>(db.d + 32);
   cudaError_t e = p->cfg.kernel == KVR_KERNEL_BULK ? launch_move_bulk(true, a, p->bulk, 1, p->sm_count, p->s_gather)
                                                    : launch_move_warp(true, a, 1, p->sm_count, p->s_gather);
   if (e != cudaSuccess) return fail(KVR_ERR_CUDA, "self-test launch: %s", cudaGetErrorString(e));
