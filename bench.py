@@ -829,6 +829,62 @@ def run_ours(args):
     group.close()
 
 
+def run_alone_by_size(args):
+    """The movers alone, launch size by launch size, beside the driver's plain device-to-device copy of the same
+    bytes (what the HBM peak is measured with).  One request with a shuffled block table is exported to / imported
+    from a device buffer (one launch each, no link involved); L2 is flushed before every launch; CUDA events; median
+    of 10 after 2 warm-ups.  Prints one JSON line (not the bench contract's)."""
+    import torch
+
+    from paper_2608_30830_b200 import kvr
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(0)
+    w = CONFIGS[args.workload]
+    L, H, D, e, BS = w.geom
+    bpt = kvr.bytes_per_token(L, H, D, e)
+    nb = (32 << 30) // (BS * bpt)                                         # 32 GiB pool
+    largest = 4 << 30
+    kernel = {"warp": kvr.KERNEL_WARP, "bulk": kvr.KERNEL_BULK}[args.kernel]
+    shape = tuple(int(x) for x in args.bulk_shape.split(",")) if args.bulk_shape else None
+    pool = kvr.Pool(L, H, D, e, BS, nb, 64 << 20, initial_free_order=free_order(SEED, nb), chunk_bytes=1 << 20,
+                    staging_slots=2, kernel=kernel, bulk_shape=shape)
+    dst = torch.empty(largest, dtype=torch.uint8, device="cuda")
+    src = torch.empty(largest, dtype=torch.uint8, device="cuda")
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    peak, peak_kind = peaks()
+    rows = []
+    for mib in (16, 64, 256, 1024, 2048, 4096):
+        nbytes = (mib << 20) // (BS * bpt) * (BS * bpt)
+        assert pool.admit(1, nbytes // bpt)[0] == kvr.OK
+        ms = {"gather": [], "scatter": [], "copy": []}
+        for it in range(12):
+            for side, fn in (("gather", pool.export_to_device), ("scatter", pool.import_from_device)):
+                flush.fill_(it)
+                torch.cuda.synchronize()
+                st, _ = fn([1], dst.data_ptr(), nbytes)
+                assert st == kvr.OK and pool.wait() == kvr.OK, kvr.last_error()
+                ms[side].append(pool.latency(1)[2])
+            flush.fill_(it)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            dst[:nbytes].copy_(src[:nbytes])
+            e1.record()
+            torch.cuda.synchronize()
+            ms["copy"].append(e0.elapsed_time(e1))
+        gbs = {k: 2 * nbytes / float(np.median(v[2:])) / 1e6 for k, v in ms.items()}
+        rows.append({"launch_mib": nbytes / 2**20, "gather_gbs": gbs["gather"], "scatter_gbs": gbs["scatter"],
+                     "plain_copy_gbs": gbs["copy"], "gather_vs_copy": gbs["gather"] / gbs["copy"],
+                     "scatter_vs_copy": gbs["scatter"] / gbs["copy"], "gather_frac_of_peak": gbs["gather"] / peak,
+                     "scatter_frac_of_peak": gbs["scatter"] / peak})
+        assert pool.release(1) == kvr.OK
+    print(json.dumps({"what": "movers alone by launch size against torch copy_ of the same bytes (GB/s of read + written bytes)",
+                      "workload_geometry": args.workload, "kernel": args.kernel, "peak": peak, "peak_kind": peak_kind, "rows": rows}))
+    pool.close()
+
+
 def relaunch_under_torchrun(args):
     """`python bench.py --gpus N` started plainly: start the N ranks (one per GPU) and pass their output through."""
     import socket
@@ -868,6 +924,8 @@ def main():
     ap.add_argument("--low-latency", action="store_true", help="batched resume with KVR_LOW_LATENCY")
     ap.add_argument("--no-share", action="store_true", help="paper_shape: every request owns its whole context")
     ap.add_argument("--no-extras", action="store_true", help="skip kernels-alone, lone-request and CPU legs")
+    ap.add_argument("--alone-by-size", action="store_true",
+                    help="the movers alone, 16 MiB to 4 GiB per launch, beside a plain device copy (its own JSON line)")
     ap.add_argument("--dry-run", action="store_true",
                     help="launcher and bookkeeping check without a GPU: metadata-only pools, gloo ranks; moves nothing")
     args = ap.parse_args()
@@ -875,6 +933,8 @@ def main():
         sys.exit(relaunch_under_torchrun(args))
     if args.impl == "reference":
         run_reference(args)
+    elif args.alone_by_size:
+        run_alone_by_size(args)
     elif args.workload == "longctx":
         run_longctx(args)
     elif args.workload == "trace":
