@@ -74,3 +74,25 @@ def test_our_arm_prints_one_contract_line_on_a_gpu():
     assert 0 < d["e2e"]["value"] <= d["value"] * 1.05 and d["gpu_launches"] >= 4
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] == 1 and d["cpu_baseline"]["value"] > 0
     assert d["host_link"]["suspend_frac_of_d2h_peak"] > 0.5 and d["host_link"]["resume_frac_of_h2d_peak"] > 0.5
+
+
+@pytest.mark.gpu
+def test_the_movers_alone_keep_up_with_a_plain_device_copy():
+    """`python bench.py --alone-by-size`: the paged gather and scatter, one launch each, beside torch's copy_ of the
+    same number of contiguous bytes.  With work handed out through the launch's counter the bulk mover is at least as
+    fast as the plain copy from 64 MiB on; the bound here is loose (shared machine), the fixed-share kernel failed it."""
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    if torch.cuda.mem_get_info()[0] < (44 << 30):
+        pytest.skip("needs 44 GiB of free device memory")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--alone-by-size"], capture_output=True, text=True,
+                         timeout=900)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [x for x in out.stdout.splitlines() if x.startswith("{")]
+    assert len(lines) == 1
+    rows = json.loads(lines[0])["rows"]
+    assert [r["launch_mib"] for r in rows] == [16, 64, 256, 1024, 2048, 4096]
+    for r in rows[3:]:
+        assert r["gather_vs_copy"] > 0.97 and r["scatter_vs_copy"] > 0.97, r
+        assert r["gather_frac_of_peak"] > 0.93 and r["scatter_frac_of_peak"] > 0.93, r
