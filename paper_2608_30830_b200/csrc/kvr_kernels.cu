@@ -99,8 +99,8 @@ __device__ __forceinline__ Tile locate(const MoveArgs &a, const long long *cum, 
 
 // ---- warp mover --------------------------------------------------------------------
 
-// One warp per tile; the warps of the grid take consecutive tiles (by the launch's work counter when there is one,
-// else grid-strided), so at any moment the grid covers one contiguous window of the image.  A lane keeps 8
+// One warp per tile; the warps of the grid take consecutive tiles from the launch's work counter, so at any moment
+// the grid covers one contiguous window of the image.  A lane keeps 8
 // independent 16-byte loads in flight (streaming cache policy: every byte is touched once) before it stores them.
 template <bool GATHER>
 __global__ void __launch_bounds__(kWarpThreads) move_warp_kernel(const MoveArgs a) {
@@ -109,25 +109,17 @@ __global__ void __launch_bounds__(kWarpThreads) move_warp_kernel(const MoveArgs 
   if (a.stamp && threadIdx.x == 0) atomicMin(a.stamp, global_ns());
   scan_segments(a, cum);
   const int lane = threadIdx.x & 31;
-  const int warps_per_cta = blockDim.x >> 5;
-  const long long stride = (long long)gridDim.x * warps_per_cta;
-  long long next = (long long)blockIdx.x * warps_per_cta + (threadIdx.x >> 5);
   // small tiles are claimed several at a time, so that the counter is not the bottleneck
   const int claim = a.tile_bytes >= kClaimBytes ? 1 : kClaimBytes / a.tile_bytes;
-  long long claim_end = 0;
+  long long next = 0, claim_end = 0;
   for (;;) {
-    long long w;
-    if (a.work) {
-      if (next >= claim_end) {
-        unsigned long long first = 0;
-        if (lane == 0) first = atomicAdd(a.work, (unsigned long long)claim);
-        next = (long long)__shfl_sync(0xffffffffu, first, 0);
-        claim_end = next + claim;
-      }
-      w = next++;
-    } else {
-      w = next; next += stride;
+    if (next >= claim_end) {
+      unsigned long long first = 0;
+      if (lane == 0) first = atomicAdd(a.work, (unsigned long long)claim);
+      next = (long long)__shfl_sync(0xffffffffu, first, 0);
+      claim_end = next + claim;
     }
+    const long long w = next++;
     if (w >= a.total_tiles) break;
     const Tile t = locate(a, cum, w);
     const uint4 *src = reinterpret_cast<const uint4 *>(GATHER ? t.pool_ptr : t.lin_ptr);
@@ -336,7 +328,7 @@ cudaError_t opt_in(size_t smem) {
 
 cudaError_t launch_move_warp(bool gather, const MoveArgs &a, int grid_limit, int sm_count, cudaStream_t s) {
   if (a.total_tiles <= 0) return cudaSuccess;
-  if (a.nsegs < 1 || a.nsegs > kMaxSegs) return cudaErrorInvalidValue;
+  if (a.nsegs < 1 || a.nsegs > kMaxSegs || !a.work) return cudaErrorInvalidValue;
   static int ctas_per_sm = 0;                     // co-resident CTAs: the grid is one full wave, never more
   if (!ctas_per_sm) {
     int n = 0;

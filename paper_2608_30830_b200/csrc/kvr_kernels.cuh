@@ -37,8 +37,7 @@ struct MoveArgs {
   unsigned long long *stamp;  // DEVICE or NULL: stamp[0] = earliest start, stamp[1] = latest end of any CTA, in
                               // %globaltimer nanoseconds (the host initialises them to ~0 and 0)
   unsigned long long *work;   // DEVICE: work counter of this launch, zero when the kernel starts.  The movers hand out
-                              // work through it (whoever is free takes the next unit), so all SMs finish together.  The
-                              // bulk mover needs it; the warp mover falls back to a grid-strided loop when it is NULL.
+                              // work through it (whoever is free takes the next unit), so all SMs finish together.
 };
 
 struct BulkShape {       // tuning of the bulk mover

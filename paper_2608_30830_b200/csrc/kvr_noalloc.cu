@@ -25,6 +25,8 @@ namespace kvr { void set_last_error(const char *msg); }
 namespace {
 
 constexpr size_t kSegBytes = 256;   // the segment record, padded so the table that follows stays 256-byte aligned
+constexpr size_t kWorkOffset = 128; // inside that padding: the launch's work counter, uploaded as zero with the record
+static_assert(sizeof(kvr::Seg) <= kWorkOffset, "the work counter would overlap the segment record");
 constexpr size_t kScratchBytes = kSegBytes + sizeof(int32_t) * (size_t)KVR_NOALLOC_MAX_BLOCKS;
 
 // Scratch of the allocation-free entry point.  In host code this name is only a handle for
@@ -106,6 +108,7 @@ extern "C" kvr_status kvr_gather_noalloc(const void *device_pool, const kvr_geom
     std::lock_guard<std::mutex> hold(g_stage_mu);
     int32_t *table = reinterpret_cast<int32_t *>(g_stage + kSegBytes);
     memcpy(g_stage, &seg, sizeof seg);
+    memset(g_stage + kWorkOffset, 0, sizeof(unsigned long long));
     memcpy(table, block_table, sizeof(int32_t) * (size_t)nb);
     for (int32_t i = 0; i < nb; ++i)
       if (table[i] < 0 || table[i] >= num_blocks) return fail_na(KVR_ERR_INVALID_ARG, "block id out of range");
@@ -127,7 +130,8 @@ extern "C" kvr_status kvr_gather_noalloc(const void *device_pool, const kvr_geom
   a.row_bytes = (int)row;
   a.block_size = g->block_size;
   a.num_blocks = num_blocks;
-  a.status = nullptr;               // the warp mover has no bounded waits and never writes it
+  a.status = nullptr;               // the warp mover has no bounded waits, and the table was checked above
+  a.work = reinterpret_cast<unsigned long long *>(scratch + kWorkOffset);
   cudaError_t e = kvr::launch_move_warp(true, a, 0, g_sm_count[dev], st);
   if (e != cudaSuccess) return fail_na(KVR_ERR_CUDA, cudaGetErrorString(e));
   return KVR_OK;
