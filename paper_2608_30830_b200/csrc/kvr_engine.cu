@@ -754,8 +754,8 @@ kvr_status create_engine(kvr_pool *p) {
       p->arena_dev = p->h_arena;
       can_map = true;
       if (at.device != c.device) {
-        // a peer's memory: make it addressable from this device (plain loads, stores and copies only -- the movers
-        // use no multicast).  "Already enabled" is fine.
+        // a peer's memory: make it addressable from this device (the movers touch it with plain loads, stores and
+        // single-CTA bulk copies only).  "Already enabled" is fine.
         cudaError_t pe = cudaDeviceEnablePeerAccess(at.device, 0);
         if (pe != cudaSuccess && pe != cudaErrorPeerAccessAlreadyEnabled) {
           cudaGetLastError();

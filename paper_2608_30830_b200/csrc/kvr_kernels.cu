@@ -11,7 +11,8 @@
 //   move_warp : one warp per tile, 16-byte loads and stores, 8 in flight per lane
 //   move_bulk : one thread per pipeline drives bulk async copies
 //               global -> shared -> global through a ring of shared-memory
-//               stages guarded by mbarriers (no multicast: no tile is shared)
+//               stages guarded by mbarriers (every copy is issued and consumed by one
+//               CTA: no tile is shared between CTAs)
 //
 // Work is handed out dynamically: a launch carries a zeroed counter and every
 // pipeline (or warp) takes the next unit (32 KiB, or a few smaller ones) with

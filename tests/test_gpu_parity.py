@@ -299,7 +299,7 @@ def test_arena_in_device_memory(route):
 @pytest.mark.parametrize("route", [kvr.ROUTE_STAGED, kvr.ROUTE_MAPPED])
 def test_arena_in_a_peer_gpus_memory(route):
     """The same with the arena on another GPU (the peer-HBM tier over NVLink): the library enables peer access, the
-    copies follow the pointer and the direct route's kernels use plain loads, stores and non-multicast bulk copies.
+    copies follow the pointer and the direct route's kernels use plain loads, stores and single-CTA bulk copies.
     Needs two GPUs: skipped on a one-GPU machine."""
     if torch.cuda.device_count() < 2:
         pytest.skip("needs two GPUs")
