@@ -386,11 +386,12 @@ def test_library_owned_pool_and_arena():
             assert np.array_equal(got[int(off):int(off) + n * bpt], host_src[int(off):int(off) + n * bpt])
 
 
+@pytest.mark.parametrize("geom", [(2, 8, 128, 2, 16), (8, 2, 128, 2, 16), (16, 1, 128, 1, 16)], ids=["tile32k", "tile8k", "tile2k"])
 @pytest.mark.parametrize("mode", [MODES[1], MODES[3], MODES[6]])
-def test_random_scripts_with_moves_that_stay_in_flight(mode):
+def test_random_scripts_with_moves_that_stay_in_flight(mode, geom):
     """The same seeded scripts on images of tens of MiB, so that calls really do arrive while earlier moves are
-    still on the link: bookkeeping as observed (including reported states) and all bytes must still equal the oracle's."""
-    geom = (2, 8, 128, 2, 16)                     # 8 KiB per token, 32 KiB tiles
+    still on the link: bookkeeping as observed (including reported states) and all bytes must still equal the oracle's.
+    Tiles of 32, 8 and 2 KiB: the movers claim one, four and sixteen units of work at a time."""
     t = Twin(geom, 2048, 300 << 20, seed=2, chunk_bytes=64 << 20, staging_slots=2, **mode)
     ops = random_script(2002, 160, max_tokens=6000, n_ids=12, batch=4)
     la, lb = run_script(t.o, ops), run_script(t.g, ops)
